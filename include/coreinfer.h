@@ -1,0 +1,214 @@
+/*
+ * coreinfer.h -- C ABI of the CoreInfer core-sparse FFN path for NVIDIA B200 (sm_100a).
+ *
+ * The library implements, on one GPU, the three stages of the method:
+ *   (1) sentence-wise core-neuron selection at pre-fill   (Definition 1 / Eq. 1,
+ *       Eq. 3, Definition 2 / Eq. 2),
+ *   (2) one-shot compaction of the selected weights       (Section 5.3: only the
+ *       needed neurons are deployed, fixed for the whole decode),
+ *   (3) the decode-stage FFN over those fixed neurons     (Section 4.2),
+ * plus a dense FFN on the uncompacted weights that produces the pre-fill
+ * activations the selection consumes.
+ *
+ * Conventions for every entry point
+ *   - "device" pointers are CUDA device memory of the current device; "host"
+ *     pointers are ordinary host memory.  Every buffer is owned by the caller.
+ *     The library allocates no device memory and keeps no state between calls
+ *     except a thread-local error string.
+ *   - Matrices are row-major and dense.  Device pointers must be 16-byte
+ *     aligned; d_model * sizeof(element) must be a multiple of 16.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *     Calls only enqueue work on that stream and return; they never
+ *     synchronise.  Outputs are valid once the stream reaches that point.
+ *   - Errors: arguments are checked on the host before anything is enqueued.
+ *     A call that returns a status other than COREINFER_OK has enqueued
+ *     nothing, except COREINFER_ERR_CUDA, which reports a failed launch.
+ *     coreinfer_last_error() gives the reason as text.  Nothing aborts, traps
+ *     or throws.
+ *   - There is no CPU fallback: without a CUDA device every compute entry point
+ *     fails with COREINFER_ERR_CUDA.
+ *   - Sizes of "top fractions" follow one rule everywhere: coreinfer_count().
+ */
+#ifndef COREINFER_H_
+#define COREINFER_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    COREINFER_OK = 0,
+    COREINFER_ERR_INVALID_ARG = 1,   /* NULL / misaligned pointer, size or fraction out of range */
+    COREINFER_ERR_UNSUPPORTED = 2,   /* dtype / kind / batch / size outside what is built */
+    COREINFER_ERR_WORKSPACE = 3,     /* workspace missing or smaller than *_workspace_bytes() */
+    COREINFER_ERR_CUDA = 4,          /* CUDA runtime reported an error (no device, failed launch) */
+    COREINFER_ERR_TIMEOUT = 5        /* a bounded device-side wait gave up (see coreinfer_workspace_status) */
+} coreinfer_status;
+
+typedef enum { COREINFER_F32 = 0, COREINFER_BF16 = 1 } coreinfer_dtype;
+
+/* FFN kinds.  RELU:        h = max(W_up x + b_up, 0)
+ *             RELU_GATED:  h = max(W_gate x, 0) * (W_up x)        (no up bias)
+ * and in both y = W_down h + b_down.  h is the "activation layer" output A(x)
+ * that Definition 1 ranks. */
+typedef enum { COREINFER_FFN_RELU = 0, COREINFER_FFN_RELU_GATED = 1 } coreinfer_ffn_kind;
+
+#define COREINFER_MAX_BATCH 8
+#define COREINFER_MAX_LAYERS 128
+
+/* Size of a "top fraction" (Definition 1: top alpha of the positive activations of
+ * a token; Definition 2: top beta of all neurons): ceil(frac * n) clamped to
+ * [0, n], evaluated as ceil(frac * n - 1e-6) in double so that decimal fractions
+ * whose product is an integer (0.2 * 20480) do not round up.  Pure host function. */
+int32_t coreinfer_count(double frac, int32_t n);
+
+/* Text of the last error on the calling thread (static storage, never NULL). */
+const char* coreinfer_last_error(void);
+
+/* ------------------------------------------------------------------ (1) --
+ * Sentence-wise core-neuron selection (Definition 1 / Eq. 1, Eq. 3,
+ * Definition 2 / Eq. 2).
+ *
+ * For each of the T rows of `act`, the token-wise core set is the
+ * k_t = coreinfer_count(alpha, P_t) largest of its P_t positive entries
+ * (positive on the bit pattern: sign clear, not zero, not NaN; equal values go
+ * to the lower index).  f[n] counts the rows whose set contains n.  The result
+ * is the K = coreinfer_count(beta, d_ff) neurons with the largest f (equal
+ * counts go to the lower index), written in ascending index order.
+ *
+ *   act         device, [T, d_ff] with row stride ld_act elements; fp32
+ *               (COREINFER_F32 only).  ld_act >= d_ff, ld_act % 4 == 0.
+ *   core_idx    device, out, K int32 (capacity >= K).
+ *   counts_out  device, out, [d_ff] int32 = f, or NULL.
+ *   workspace   device scratch of at least coreinfer_select_workspace_bytes();
+ *               contents need not be initialised and are clobbered.
+ * Errors: INVALID_ARG (NULL, alignment, T < 1, d_ff < 1, alpha or beta outside
+ * (0, 1]), UNSUPPORTED (dtype; d_ff or T beyond what the kernels are built
+ * for, see coreinfer_last_error), WORKSPACE, CUDA. */
+size_t coreinfer_select_workspace_bytes(int32_t T, int32_t d_ff);
+
+coreinfer_status coreinfer_select_core(const void* act, coreinfer_dtype act_dtype,
+                                       int32_t T, int32_t d_ff, int64_t ld_act,
+                                       double alpha, double beta,
+                                       int32_t* core_idx, int32_t* counts_out,
+                                       void* workspace, size_t workspace_bytes,
+                                       void* cuda_stream);
+
+/* ------------------------------------------------------------------ (2) --
+ * Compaction (Section 5.3: the neurons found at pre-fill are the only ones
+ * deployed for decoding).  Pure data movement; outputs are byte-identical
+ * copies of the selected elements.
+ *
+ *   w_up    device [d_ff, d_model]          w_up_c    device out [K, d_model]  = w_up[core_idx[k], :]
+ *   w_gate  device [d_ff, d_model] or NULL  w_gate_c  device out [K, d_model]  (NULL iff w_gate NULL)
+ *   w_down  device [d_model, d_ff]          w_downT_c device out [K, d_model]  = w_down[:, core_idx[k]]
+ *   b_up    device [d_ff] or NULL           b_up_c    device out [K]           (NULL iff b_up NULL)
+ *   core_idx device [K] int32, ascending, unique, each in [0, d_ff) (trusted).
+ * All tensors share `dtype`.  1 <= K <= d_ff.
+ * Errors: INVALID_ARG, UNSUPPORTED, CUDA. */
+coreinfer_status coreinfer_compact(const void* w_up, const void* w_gate, const void* w_down,
+                                   const void* b_up, coreinfer_dtype dtype,
+                                   int32_t d_model, int32_t d_ff,
+                                   const int32_t* core_idx, int32_t K,
+                                   void* w_up_c, void* w_gate_c, void* w_downT_c, void* b_up_c,
+                                   void* cuda_stream);
+
+/* ------------------------------------------------------------------ (3) --
+ * Decode FFN over compacted weights (Section 4.2), one layer:
+ *   h_k = act(w_up_c[k,:] . x (+ b_up_c[k]))   [gated: max(w_gate_c[k,:] . x, 0) * (w_up_c[k,:] . x)]
+ *   y_j = sum_k h_k * w_downT_c[k, j] + b_down[j]
+ * h is held in fp32 and never leaves the chip (Section 5 "Models": fp32
+ * intermediate activations).  Sums are fp32; their order is not fixed between
+ * runs (partial results are combined with floating-point atomics).
+ *
+ *   x          device [batch, d_model] in `dtype`
+ *   w_*_c      device [K, d_model] in `dtype` (w_gate_c NULL iff kind is RELU)
+ *   b_up_c     device [K] in `dtype` or NULL (RELU only); b_down device [d_model] in `dtype` or NULL
+ *   y          device out [batch, d_model] fp32
+ *   workspace  device scratch of at least coreinfer_ffn_decode_workspace_bytes().
+ * 1 <= batch <= COREINFER_MAX_BATCH.
+ * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA. */
+size_t coreinfer_ffn_decode_workspace_bytes(int32_t batch, int32_t d_model, int32_t K);
+
+coreinfer_status coreinfer_ffn_decode(const void* x, int32_t batch, coreinfer_dtype dtype,
+                                      coreinfer_ffn_kind kind, int32_t d_model, int32_t K,
+                                      const void* w_up_c, const void* w_gate_c,
+                                      const void* w_downT_c,
+                                      const void* b_up_c, const void* b_down,
+                                      float* y, void* workspace, size_t workspace_bytes,
+                                      void* cuda_stream);
+
+/* One decode step through a stack of L compacted FFN layers in a single
+ * persistent launch (the decode loop of Section 4.2 over all layers: the sets are
+ * fixed, so every layer's weights can be streamed without waiting for its input).
+ * The paper does not describe what sits between two FFN layers; this entry point
+ * chains them with a parameter-free residual + RMS normalisation,
+ *   x_{l+1} = round_to_dtype( (x_l + y_l) / sqrt(mean_j (x_l + y_l)_j^2) ),
+ * so that each layer truly depends on the previous one.
+ *
+ *   layers     host array of L descriptors (device pointers inside, same meaning
+ *              as in coreinfer_ffn_decode); read during the call only.
+ *   x0         device [batch, d_model] in `dtype`: input of layer 0.
+ *   y_last     device out [batch, d_model] fp32: FFN output of layer L-1.
+ *   y_layers   device out [L, batch, d_model] fp32: every layer's FFN output, or NULL.
+ *   x_layers   device out [L, batch, d_model] in `dtype`: every layer's input as
+ *              consumed, or NULL.
+ *   workspace  at least coreinfer_ffn_decode_stack_workspace_bytes().
+ * batch must be 1.  1 <= L <= COREINFER_MAX_LAYERS.
+ * Thread blocks of this launch wait on one another at layer boundaries; every
+ * such wait is bounded, and a wait that gives up makes all blocks return early
+ * and records COREINFER_ERR_TIMEOUT in the workspace (read it with
+ * coreinfer_workspace_status after the stream has drained).  The launch is
+ * cooperative: it needs the whole GPU to itself to be co-resident.
+ * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA. */
+typedef struct {
+    const void* w_up_c;
+    const void* w_gate_c;
+    const void* w_downT_c;
+    const void* b_up_c;
+    const void* b_down;
+    int32_t K;
+    int32_t reserved;
+} coreinfer_layer;
+
+size_t coreinfer_ffn_decode_stack_workspace_bytes(int32_t L, int32_t batch, int32_t d_model,
+                                                  int32_t K_max);
+
+coreinfer_status coreinfer_ffn_decode_stack(const coreinfer_layer* layers, int32_t L,
+                                            const void* x0, int32_t batch,
+                                            coreinfer_dtype dtype, coreinfer_ffn_kind kind,
+                                            int32_t d_model,
+                                            float* y_last, float* y_layers, void* x_layers,
+                                            void* workspace, size_t workspace_bytes,
+                                            void* cuda_stream);
+
+/* Synchronises `cuda_stream`, then reads the status word that the most recent
+ * decode call using `workspace` left there: COREINFER_OK, or COREINFER_ERR_TIMEOUT
+ * if a bounded device-side wait gave up (outputs of that call are then
+ * undefined).  Returns COREINFER_ERR_CUDA if the synchronisation or copy fails. */
+coreinfer_status coreinfer_workspace_status(const void* workspace, void* cuda_stream);
+
+/* ------------------------------------------------------------------ (4) --
+ * Dense FFN on the uncompacted weights: the pre-fill pass whose intermediate
+ * activations A = h [T, d_ff] are what Definition 1 is applied to.
+ *
+ *   x       device [T, d_model] in `dtype`
+ *   w_up    device [d_ff, d_model]; w_gate same or NULL (NULL iff RELU); w_down device [d_model, d_ff]
+ *   b_up    device [d_ff] or NULL (RELU only); b_down device [d_model] or NULL; all in `dtype`
+ *   h_out   device out [T, d_ff] fp32 or NULL
+ *   y_out   device out [T, d_model] fp32 or NULL (needs h_out: y is computed from the stored fp32 h)
+ * Products are exact (fp32 or bf16 inputs), sums are fp32.
+ * Errors: INVALID_ARG, UNSUPPORTED, CUDA. */
+coreinfer_status coreinfer_ffn_dense_ref(const void* x, int32_t T, coreinfer_dtype dtype,
+                                         coreinfer_ffn_kind kind, int32_t d_model, int32_t d_ff,
+                                         const void* w_up, const void* w_gate, const void* w_down,
+                                         const void* b_up, const void* b_down,
+                                         float* h_out, float* y_out, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* COREINFER_H_ */

@@ -1,0 +1,453 @@
+// Sentence-wise core-neuron selection at pre-fill (Definition 1 / Eq. 1, Eq. 3,
+// Definition 2 / Eq. 2).  Three kernels, all integer work on float bit patterns, so the
+// result is exact and independent of scheduling:
+//
+//   select_rows_kernel   persistent CTAs, each walks rows t = cta, cta + G, ...  A row is
+//                        brought into shared memory by bulk copies (the next row is
+//                        prefetched when two rows fit).  Per row: count the positives P,
+//                        k = ceil(alpha P), then an MSB-first radix select (12 + 12 + 7 bits)
+//                        finds the exact bit pattern of the k-th largest positive value and
+//                        how many entries equal to it are admitted (lowest index first).
+//                        Each thread owns fixed columns of every row, so the per-neuron
+//                        membership counters of Eq. 3 live in its registers: no atomics.
+//                        At the end each CTA writes its counters as one u16 row.
+//   select_count_kernel  f[n] = sum over CTAs of those rows (int32).
+//   select_top_kernel    one CTA: the K-th largest count c* by bisection on the count value,
+//                        then an index-ordered scan admits f > c*, and the lowest-index
+//                        f == c* until K are taken, and writes them in ascending index.
+#include "common.cuh"
+
+namespace coreinfer {
+
+constexpr int kSelThreads = 1024;
+constexpr int kSelWarps = kSelThreads / 32;
+constexpr int kSelMaxCtas = 256;
+constexpr int kSelMaxVpt = 9;                        // d_ff <= 9 * 1024 * 4 = 36864
+constexpr int kSelBins = 4096;
+constexpr int kSelCtrlBytes = 256;
+constexpr uint32_t kCopyChunk = 32768;
+constexpr long long kSelWaitCycles = 3000000000LL;
+
+// ceil(alpha * P - 1e-6) clamped to [0, P]; same expression as coreinfer_count, with the
+// product and the difference rounded separately (no contraction).
+__device__ __forceinline__ int count_dev(double frac, int n)
+{
+    if (n <= 0) return 0;
+    double c = ceil(__dsub_rn(__dmul_rn(frac, (double)n), 1e-6));
+    if (c < 0.0) c = 0.0;
+    if (c > (double)n) c = (double)n;
+    return (int)c;
+}
+
+__device__ __forceinline__ bool is_pos_bits(uint32_t b) { return (b - 1u) < 0x7F800000u; }
+
+struct SelShared {
+    int warp_tot[kSelWarps];
+    int bin, above, bin_count, total;
+    int abort_flag;
+};
+
+// Exclusive prefix sum over the block's threads; *total gets the block sum.
+__device__ __forceinline__ int block_excl_scan(int v, SelShared* sh, int* total)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    if (lane == 31) sh->warp_tot[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        int w = sh->warp_tot[lane];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int t = __shfl_up_sync(0xffffffffu, w, o);
+            if (lane >= o) w += t;
+        }
+        sh->warp_tot[lane] = w;
+    }
+    __syncthreads();
+    const int base = warp > 0 ? sh->warp_tot[warp - 1] : 0;
+    *total = sh->warp_tot[kSelWarps - 1];
+    __syncthreads();
+    return base + incl - v;
+}
+
+// hist[kSelBins] holds digit counts.  Finds the bin holding the k-th largest element
+// (1 <= k <= total): sh->bin, sh->above = elements in higher bins, sh->bin_count.
+// With k_from_total, k = ceil(alpha * total) is formed here (total = number of positives).
+// Returns k (block-uniform); with k == 0 nothing else is written.
+__device__ __forceinline__ int find_bin(const int* hist, int k, bool k_from_total, double alpha,
+                                        SelShared* sh)
+{
+    constexpr int PER = kSelBins / kSelThreads;   // 4 bins per thread, walked from the top
+    const int top = kSelBins - 1 - PER * (int)threadIdx.x;
+    int c[PER], s = 0;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) { c[i] = hist[top - i]; s += c[i]; }
+    int total;
+    const int before = block_excl_scan(s, sh, &total);
+    if (k_from_total) k = count_dev(alpha, total);
+    if (k > 0 && before < k && k <= before + s) {
+        int above = before;
+#pragma unroll
+        for (int i = 0; i < PER; ++i) {
+            if (above < k && k <= above + c[i]) { sh->bin = top - i; sh->above = above; sh->bin_count = c[i]; }
+            above += c[i];
+        }
+    }
+    __syncthreads();
+    return k;
+}
+
+// HOLD: the thread keeps its columns of the row in registers (the shared-memory buffer is
+// free for the next row at once); otherwise every pass re-reads them from shared memory.
+template <int VPT, bool HOLD>
+__global__ void __launch_bounds__(kSelThreads, 1)
+select_rows_kernel(const float* __restrict__ act, int T, int N, long long ld, double alpha,
+                   uint16_t* __restrict__ partial, unsigned* __restrict__ status, int nbuf, int row_bytes)
+{
+    extern __shared__ __align__(128) uint8_t smem[];
+    const int buf_bytes = (row_bytes + 127) & ~127;
+    int* hist = reinterpret_cast<int*>(smem + (size_t)nbuf * buf_bytes);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(hist + kSelBins);   // [2]
+    SelShared* sh = reinterpret_cast<SelShared*>(bars + 2);
+
+    const int tid = threadIdx.x;
+    const int G = gridDim.x;
+    const int nvec = row_bytes / 16;
+
+    if (tid == 0) {
+        mbar_init(smem_u32(&bars[0]), 1);
+        mbar_init(smem_u32(&bars[1]), 1);
+        sh->abort_flag = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+
+    int issued[2] = {0, 0};                // thread 0: copies issued per buffer
+    auto issue_row = [&](int t, int b) {   // thread 0 only
+        const uint32_t bar = smem_u32(&bars[b]);
+        mbar_arrive_expect_tx(bar, (uint32_t)row_bytes);
+        const uint8_t* src = reinterpret_cast<const uint8_t*>(act + (long long)t * ld);
+        const uint32_t dst = smem_u32(smem + (size_t)b * buf_bytes);
+        for (uint32_t off = 0; off < (uint32_t)row_bytes; off += kCopyChunk) {
+            const uint32_t n = min(kCopyChunk, (uint32_t)row_bytes - off);
+            bulk_g2s(dst + off, src + off, n, bar);
+        }
+        ++issued[b];
+    };
+
+    int cnt[VPT][4];
+#pragma unroll
+    for (int i = 0; i < VPT; ++i)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) cnt[i][e] = 0;
+
+    if (tid == 0 && (int)blockIdx.x < T) issue_row(blockIdx.x, 0);
+
+    int iter = 0;
+    for (int t = blockIdx.x; t < T; t += G, ++iter) {
+        const int b = (nbuf == 2) ? (iter & 1) : 0;
+        const uint32_t parity = (nbuf == 2) ? ((iter >> 1) & 1) : (iter & 1);
+        // every thread finished with the previous row (barrier at the end of the loop body)
+        if (tid == 0) {
+            if (nbuf == 2) { if (t + G < T) issue_row(t + G, b ^ 1); }
+            else if (!HOLD && iter > 0) issue_row(t, 0);
+        }
+
+        {   // bounded wait for this row's bytes
+            const uint32_t bar = smem_u32(&bars[b]);
+            if (!mbar_try_wait(bar, parity)) {
+                const long long t0 = clock64();
+                while (!mbar_try_wait(bar, parity)) {
+                    if (clock64() - t0 > kSelWaitCycles) {
+                        sh->abort_flag = 1;
+                        atomicMax(status, (unsigned)kStatusTimeout);
+                        break;
+                    }
+                }
+            }
+        }
+        __syncthreads();
+        if (sh->abort_flag) break;   // block-uniform
+
+        const uint4* row = reinterpret_cast<const uint4*>(smem + (size_t)b * buf_bytes);
+        // masked bit patterns of vector i: 0 stands for "not positive" (or beyond d_ff)
+        auto load_vec = [&](int i) -> uint4 {
+            const int v = tid + i * kSelThreads;
+            uint4 q = make_uint4(0, 0, 0, 0);
+            if (v < nvec) q = row[v];
+            if (v * 4 + 0 >= N || !is_pos_bits(q.x)) q.x = 0u;
+            if (v * 4 + 1 >= N || !is_pos_bits(q.y)) q.y = 0u;
+            if (v * 4 + 2 >= N || !is_pos_bits(q.z)) q.z = 0u;
+            if (v * 4 + 3 >= N || !is_pos_bits(q.w)) q.w = 0u;
+            return q;
+        };
+        uint4 held[HOLD ? VPT : 1];
+        if (HOLD) {
+#pragma unroll
+            for (int i = 0; i < VPT; ++i) held[i] = load_vec(i);
+            __syncthreads();   // every thread holds its columns: the buffer may be refilled
+            if (nbuf == 1 && tid == 0 && t + G < T) issue_row(t + G, 0);
+        }
+        auto vec = [&](int i) -> uint4 { return HOLD ? held[HOLD ? i : 0] : load_vec(i); };
+
+        // ---- radix select of the k-th largest positive pattern: 12 + 12 + 7 bits ----
+        uint32_t vstar = 0u;
+        int need = 0, eq_total = 0;
+#pragma unroll 1
+        for (int pass = 0; pass < 3; ++pass) {
+            const int shift = pass == 0 ? 19 : (pass == 1 ? 7 : 0);
+            const uint32_t dmask = pass == 2 ? 0x7Fu : 0xFFFu;
+            const int pshift = pass == 0 ? 31 : (pass == 1 ? 19 : 7);   // prefix = bits >> pshift
+            for (int i = tid; i < kSelBins; i += kSelThreads) hist[i] = 0;
+            __syncthreads();
+#pragma unroll
+            for (int i = 0; i < VPT; ++i) {
+                const uint4 q = vec(i);
+                const uint32_t bb[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (bb[e] != 0u && (bb[e] >> pshift) == (vstar >> pshift))
+                        atomicAdd(&hist[(bb[e] >> shift) & dmask], 1);
+            }
+            __syncthreads();
+            need = find_bin(hist, need, pass == 0, alpha, sh);
+            if (need == 0) break;                      // no positive entry in this row
+            vstar |= (uint32_t)sh->bin << shift;
+            need -= sh->above;
+            eq_total = sh->bin_count;
+            __syncthreads();
+        }
+
+        // ---- membership (Eq. 1) and its count (Eq. 3) ----
+        if (need == 0) {
+            // nothing to count
+        } else if (need == eq_total) {
+#pragma unroll
+            for (int i = 0; i < VPT; ++i) {
+                const uint4 q = vec(i);
+                cnt[i][0] += (q.x >= vstar) ? 1 : 0;   // vstar > 0, masked entries are 0
+                cnt[i][1] += (q.y >= vstar) ? 1 : 0;
+                cnt[i][2] += (q.z >= vstar) ? 1 : 0;
+                cnt[i][3] += (q.w >= vstar) ? 1 : 0;
+            }
+        } else {
+            // more entries equal the threshold than places left: lower index first.
+            // Index order = vector round i, then thread, then element.
+            int taken = 0;
+#pragma unroll
+            for (int i = 0; i < VPT; ++i) {
+                const uint4 q = vec(i);
+                const uint32_t bb[4] = {q.x, q.y, q.z, q.w};
+                int c = 0;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) c += (bb[e] == vstar) ? 1 : 0;
+                int tot;
+                int rank = taken + block_excl_scan(c, sh, &tot);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    if (bb[e] > vstar) cnt[i][e] += 1;
+                    else if (bb[e] == vstar) { cnt[i][e] += (rank < need) ? 1 : 0; ++rank; }
+                }
+                taken += tot;
+            }
+        }
+        __syncthreads();   // the row buffer and the shared scratch are free again
+    }
+
+    // Never leave with a copy into this CTA's shared memory in flight.  On the normal path
+    // every issued copy has been waited for; after an abort this is a last bounded wait.
+    __syncthreads();
+    if (tid == 0) {
+        for (int b = 0; b < 2; ++b) {
+            if (issued[b] == 0) continue;
+            const uint32_t ph = (uint32_t)((issued[b] - 1) & 1);
+            const long long t0 = clock64();
+            while (!mbar_try_wait(smem_u32(&bars[b]), ph))
+                if (clock64() - t0 > kSelWaitCycles) { atomicMax(status, (unsigned)kStatusTimeout); break; }
+        }
+    }
+
+    uint16_t* out = partial + (size_t)blockIdx.x * ((size_t)nvec * 4);
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+        const int v = tid + i * kSelThreads;
+        if (v < nvec) {
+            uint2 w;
+            w.x = (uint32_t)cnt[i][0] | ((uint32_t)cnt[i][1] << 16);
+            w.y = (uint32_t)cnt[i][2] | ((uint32_t)cnt[i][3] << 16);
+            reinterpret_cast<uint2*>(out)[v] = w;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(256)
+select_count_kernel(const uint16_t* __restrict__ partial, int G, int n4, int N, int32_t* __restrict__ f)
+{
+    const int v = blockIdx.x * blockDim.x + threadIdx.x;   // one group of 4 neurons per thread
+    if (v * 4 >= N) return;
+    int c0 = 0, c1 = 0, c2 = 0, c3 = 0;
+    for (int g = 0; g < G; ++g) {
+        const uint2 w = reinterpret_cast<const uint2*>(partial + (size_t)g * n4)[v];
+        c0 += w.x & 0xffff; c1 += w.x >> 16; c2 += w.y & 0xffff; c3 += w.y >> 16;
+    }
+    const int n = v * 4;
+    f[n] = c0;
+    if (n + 1 < N) f[n + 1] = c1;
+    if (n + 2 < N) f[n + 2] = c2;
+    if (n + 3 < N) f[n + 3] = c3;
+}
+
+// One CTA.  Thread t owns the contiguous neurons [t*C, (t+1)*C).
+__global__ void __launch_bounds__(kSelThreads, 1)
+select_top_kernel(const int32_t* __restrict__ f, int N, int K, int T, int32_t* __restrict__ S)
+{
+    extern __shared__ __align__(128) uint8_t smem[];
+    int* fs = reinterpret_cast<int*>(smem);                               // [N]
+    SelShared* sh = reinterpret_cast<SelShared*>(fs + ((N + 3) & ~3));
+    const int tid = threadIdx.x;
+    for (int i = tid; i < N; i += kSelThreads) fs[i] = f[i];
+    __syncthreads();
+    const int C = (N + kSelThreads - 1) / kSelThreads;
+    const int n0 = min(tid * C, N), n1 = min(n0 + C, N);
+
+    // c* = smallest c with #(f > c) < K  (the K-th largest count), by bisection on [0, T]
+    int lo = 0, hi = T;                 // invariant: #(f > hi) < K (counts never exceed T)
+    int above_hi = 0;
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        int c = 0;
+        for (int n = n0; n < n1; ++n) c += fs[n] > mid ? 1 : 0;
+        int tot;
+        block_excl_scan(c, sh, &tot);
+        if (tot < K) { hi = mid; above_hi = tot; } else { lo = mid + 1; }
+    }
+    const int cstar = lo;
+    {   // #(f > c*) (above_hi is stale if the loop never lowered hi to c*)
+        int c = 0;
+        for (int n = n0; n < n1; ++n) c += fs[n] > cstar ? 1 : 0;
+        block_excl_scan(c, sh, &above_hi);
+    }
+    const int need = K - above_hi;      // how many f == c* are admitted, lowest index first
+
+    int ce = 0;
+    for (int n = n0; n < n1; ++n) ce += fs[n] == cstar ? 1 : 0;
+    int tot;
+    int rank = block_excl_scan(ce, sh, &tot);
+    int cm = 0;
+    {
+        int r = rank;
+        for (int n = n0; n < n1; ++n) {
+            const int v = fs[n];
+            if (v > cstar) ++cm;
+            else if (v == cstar) { cm += (r < need) ? 1 : 0; ++r; }
+        }
+    }
+    int pos = block_excl_scan(cm, sh, &tot);
+    for (int n = n0; n < n1; ++n) {
+        const int v = fs[n];
+        bool m = v > cstar;
+        if (v == cstar) { m = rank < need; ++rank; }
+        if (m) S[pos++] = n;
+    }
+}
+
+static size_t sel_fixed_smem() { return kSelBins * sizeof(int) + 2 * sizeof(uint64_t) + sizeof(SelShared) + 128; }
+
+template <int VPT>
+static coreinfer_status launch_rows(int grid, size_t smem, cudaStream_t st, const float* act, int T, int N,
+                                    long long ld, double alpha, uint16_t* partial, unsigned* status, int nbuf,
+                                    int row_bytes)
+{
+    auto kern = select_rows_kernel<VPT, (VPT <= 5)>;
+    CI_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    kern<<<grid, kSelThreads, smem, st>>>(act, T, N, ld, alpha, partial, status, nbuf, row_bytes);
+    CI_CUDA(cudaGetLastError());
+    return COREINFER_OK;
+}
+
+}  // namespace coreinfer
+
+using namespace coreinfer;
+
+extern "C" {
+
+size_t coreinfer_select_workspace_bytes(int32_t T, int32_t d_ff)
+{
+    if (T < 1 || d_ff < 1) return 0;
+    const size_t n4 = ((size_t)d_ff + 3) & ~(size_t)3;
+    const size_t ctas = (size_t)(T < kSelMaxCtas ? T : kSelMaxCtas);
+    return kSelCtrlBytes + ctas * n4 * sizeof(uint16_t) + n4 * sizeof(int32_t);
+}
+
+coreinfer_status coreinfer_select_core(const void* act, coreinfer_dtype act_dtype, int32_t T, int32_t d_ff,
+                                       int64_t ld_act, double alpha, double beta, int32_t* core_idx,
+                                       int32_t* counts_out, void* workspace, size_t workspace_bytes,
+                                       void* cuda_stream)
+{
+    if (act_dtype != COREINFER_F32)
+        CI_FAIL(COREINFER_ERR_UNSUPPORTED, "activations must be fp32 (dtype %d given)", (int)act_dtype);
+    if (!act || !core_idx) CI_FAIL(COREINFER_ERR_INVALID_ARG, "act / core_idx is NULL");
+    if (T < 1 || d_ff < 1) CI_FAIL(COREINFER_ERR_INVALID_ARG, "T = %d, d_ff = %d must be >= 1", T, d_ff);
+    if (!(alpha > 0.0 && alpha <= 1.0) || !(beta > 0.0 && beta <= 1.0))
+        CI_FAIL(COREINFER_ERR_INVALID_ARG, "alpha = %g, beta = %g must lie in (0, 1]", alpha, beta);
+    if (ld_act < d_ff || (ld_act & 3) != 0 || !aligned16(act))
+        CI_FAIL(COREINFER_ERR_INVALID_ARG, "act must be 16-byte aligned with ld_act >= d_ff and ld_act %% 4 == 0");
+    if (d_ff > kSelMaxVpt * kSelThreads * 4)
+        CI_FAIL(COREINFER_ERR_UNSUPPORTED, "d_ff = %d exceeds %d", d_ff, kSelMaxVpt * kSelThreads * 4);
+    if (!workspace || !aligned16(workspace)) CI_FAIL(COREINFER_ERR_WORKSPACE, "workspace is NULL or misaligned");
+    const size_t need = coreinfer_select_workspace_bytes(T, d_ff);
+    if (workspace_bytes < need)
+        CI_FAIL(COREINFER_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, need);
+    DeviceInfo di;
+    coreinfer_status s = device_info(&di);
+    if (s != COREINFER_OK) return s;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+
+    const int n4 = (d_ff + 3) & ~3;
+    const int row_bytes = n4 * 4;
+    int G = T < di.sm_count ? T : di.sm_count;
+    if (G > kSelMaxCtas) G = kSelMaxCtas;
+    if ((T + G - 1) / G > 65535)
+        CI_FAIL(COREINFER_ERR_UNSUPPORTED, "T = %d: more than 65535 rows per CTA", T);
+    const int K = coreinfer_count(beta, d_ff);
+
+    unsigned* status = (unsigned*)workspace;
+    uint16_t* partial = (uint16_t*)((uint8_t*)workspace + kSelCtrlBytes);
+    int32_t* f = counts_out ? counts_out : (int32_t*)(partial + (size_t)(T < kSelMaxCtas ? T : kSelMaxCtas) * n4);
+    CI_CUDA(cudaMemsetAsync(workspace, 0, kSelCtrlBytes, st));
+
+    const size_t buf = ((size_t)row_bytes + 127) & ~(size_t)127;
+    const size_t fixed = sel_fixed_smem();
+    if (fixed + buf > (size_t)di.smem_optin)
+        CI_FAIL(COREINFER_ERR_UNSUPPORTED, "a row of d_ff = %d does not fit in shared memory", d_ff);
+    const int nbuf = (fixed + 2 * buf <= (size_t)di.smem_optin) ? 2 : 1;
+    const size_t smem = fixed + nbuf * buf;
+    const int vpt = (n4 / 4 + kSelThreads - 1) / kSelThreads;
+#define CI_ROWS(V)                                                                                        \
+    case V:                                                                                               \
+        s = launch_rows<V>(G, smem, st, (const float*)act, T, d_ff, (long long)ld_act, alpha, partial,    \
+                           status, nbuf, row_bytes);                                                      \
+        break;
+    switch (vpt) {
+        CI_ROWS(1) CI_ROWS(2) CI_ROWS(3) CI_ROWS(4) CI_ROWS(5) CI_ROWS(6) CI_ROWS(7) CI_ROWS(8) CI_ROWS(9)
+        default: CI_FAIL(COREINFER_ERR_UNSUPPORTED, "d_ff = %d not built", d_ff);
+    }
+#undef CI_ROWS
+    if (s != COREINFER_OK) return s;
+
+    select_count_kernel<<<(n4 / 4 + 255) / 256, 256, 0, st>>>(partial, G, n4, d_ff, f);
+    CI_CUDA(cudaGetLastError());
+
+    const size_t smem_top = (size_t)n4 * sizeof(int) + sizeof(SelShared) + 16;
+    CI_CUDA(cudaFuncSetAttribute(select_top_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_top));
+    select_top_kernel<<<1, kSelThreads, smem_top, st>>>(f, d_ff, K, T, core_idx);
+    CI_CUDA(cudaGetLastError());
+    return COREINFER_OK;
+}
+
+}  // extern "C"
