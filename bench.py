@@ -1,0 +1,413 @@
+#!/usr/bin/env python
+"""Benchmark of the core-sparse FFN path: tokens/s of the whole request (selection +
+compaction + batch-1 decode through all layers) on synthetic, model-shaped data.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl reference]
+
+One "step" is one request: per layer, core-neuron selection on the resident pre-fill
+activations and compaction of the selected weights, then `decode_steps` batch-1 tokens, each
+one launch through all compacted layers.  Rank 0 prints ONE JSON line.
+
+--impl reference times the CPU oracle, as it stands, on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "core-sparse decode tokens/s at batch 1; achieved HBM GB/s vs B200 peak"
+UNIT = "tokens/s"
+FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode_stack_kernel launch at the bench
+# workload, from the ncu capture summarised in profiles/ (None until captured for this kernel)
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", default="opt6.7b")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-dense", action="store_true", help="skip the dense (alpha = beta = 1) comparison")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ------------------------------------------------------------------ clocks ---
+class ClockSampler(threading.Thread):
+    """Samples SM clock and clock-event reasons of one GPU through NVML while the timed region runs."""
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
+               0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown"}
+
+    def __init__(self, torch_device_index: int, period_s: float = 0.05):
+        super().__init__(daemon=True)
+        self.period = period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.handle = None
+        try:
+            import pynvml
+            import torch
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            try:
+                uuid = "GPU-" + str(torch.cuda.get_device_properties(torch_device_index).uuid)
+                self.handle = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                self.handle = pynvml.nvmlDeviceGetHandleByIndex(torch_device_index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.handle = None
+
+    def run(self):
+        if self.handle is None:
+            return
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(int(self.nv.nvmlDeviceGetClockInfo(self.handle, self.nv.NVML_CLOCK_SM)))
+                try:
+                    mask = int(self.nv.nvmlDeviceGetCurrentClocksEventReasons(self.handle))
+                except Exception:
+                    mask = int(self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle))
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop_evt.wait(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2.0)
+        s = sorted(self.samples)
+        return {"sm_mhz": (s[len(s) // 2] if s else None), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(s)}
+
+
+# ------------------------------------------------------------- CPU baseline ---
+def host_activations(cfg, X, w_up, w_gate):
+    """Input of the CPU baseline's selection: the layer's pre-fill activations [T, d_ff] fp32, made
+    with torch's CPU matmul (input generation, neither the oracle nor the CUDA path)."""
+    import torch
+    u = X.float() @ w_up.float().t()
+    if cfg.gated:
+        return (torch.relu(X.float() @ w_gate.float().t()) * u).numpy()
+    return torch.relu(u).numpy()
+
+
+def reduce_max(value: float, device=None) -> float:
+    """Max over ranks of a host scalar (identity without a process group)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tokens_per_s(world: int, steps: int, tokens_per_step: int, max_ms: float) -> float:
+    """Every rank serves its own requests (no data-path collective): units of all ranks / slowest rank's time."""
+    return world * steps * tokens_per_step / (max_ms * 1e-3)
+
+
+def oracle_sample(cfg, n_layers=2, n_tokens=4, seed_layer=0):
+    """Times the oracle on a bounded sample of the workload: selection + compaction of `n_layers`
+    layers (full T, d_ff) and `n_tokens` decode tokens through those layers (with the glue),
+    then scales to the whole request: L layers, cfg.decode_steps tokens.  Returns tokens/s."""
+    import numpy as np
+    import torch
+    import oracle
+    from paper_2410_18311_b200 import workloads as wl
+
+    f32 = lambda t: None if t is None else t.float().numpy()
+    kind = oracle.RELU_GATED if cfg.gated else oracle.RELU
+    X = wl.prompt_hidden(cfg, device="cpu")
+    t_select = t_compact = t_decode = 0.0
+    layers = []
+    for l in range(n_layers):
+        w_up, w_gate, w_down = wl.layer_weights(cfg, seed_layer + l, device="cpu")
+        H = host_activations(cfg, X, w_up, w_gate)                                    # untimed input
+        t0 = time.perf_counter()
+        S, _ = oracle.select(H, cfg.alpha, cfg.beta)
+        t1 = time.perf_counter()
+        raw = lambda t: None if t is None else (t.view(torch.int16).numpy() if t.dtype == torch.bfloat16 else t.numpy())
+        up_c, gate_c, down_c, _ = oracle.compact(raw(w_up), raw(w_gate), raw(w_down), None, S)
+        t2 = time.perf_counter()
+        t_select += t1 - t0
+        t_compact += t2 - t1
+        back = lambda a: None if a is None else (torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).float().numpy()
+                                                if cfg.dtype == "bf16" else a)
+        layers.append((back(up_c), back(gate_c), back(down_c)))
+    for tok in range(n_tokens):
+        x = f32(wl.decode_input(cfg, tok, device="cpu"))
+        t0 = time.perf_counter()
+        for (up_c, gate_c, down_c) in layers:
+            y = oracle.ffn(x, kind, up_c, gate_c, down_c)
+            x = torch.from_numpy(oracle.glue(x, y)).to(cfg.torch_dtype).float().numpy()[None, :]
+        t_decode += time.perf_counter() - t0
+    per_layer_prefill = (t_select + t_compact) / n_layers
+    per_token = t_decode / n_tokens / n_layers * cfg.L
+    request_s = per_layer_prefill * cfg.L + per_token * cfg.decode_steps
+    return {
+        "value": cfg.decode_steps / request_s, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+        "sample": "%d of %d layers (selection T=%d + compaction) and %d decode tokens through them, scaled "
+                  "linearly to %d layers x %d tokens" % (n_layers, cfg.L, cfg.T, n_tokens, cfg.L, cfg.decode_steps),
+        "select_ms_per_layer": 1e3 * t_select / n_layers, "compact_ms_per_layer": 1e3 * t_compact / n_layers,
+        "decode_ms_per_token": 1e3 * per_token, "sample_seconds": t_select + t_compact + t_decode,
+    }
+
+
+def run_reference(args, cfg):
+    """--impl reference: the oracle on host cores; each step is one bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample(cfg, n_layers=1, n_tokens=1)
+    vals, t0 = [], time.perf_counter()
+    last = None
+    for _ in range(args.steps):
+        last = oracle_sample(cfg, n_layers=1, n_tokens=2)
+        vals.append(last["value"])
+    wall = time.perf_counter() - t0
+    v = sum(vals) / len(vals)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * cfg.decode_steps / v, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
+        "config": {"workload": cfg.name, "L": cfg.L, "d_model": cfg.d_model, "d_ff": cfg.d_ff, "T": cfg.T,
+                   "alpha": cfg.alpha, "beta": cfg.beta, "decode_steps": cfg.decode_steps, "batch": 1},
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": last["cores"], "kind": "oracle", "sample": last["sample"]},
+        "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0, "wall_s": wall,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------- GPU arm ----
+def prefill_inputs(ci, wl, cfg, device):
+    """Synthetic request state resident in HBM: dense weights of every layer and the fp32
+    pre-fill activations A[l] = [T, d_ff] (dense FFN chained through the layers with the same
+    residual + RMS glue the decode stack uses)."""
+    import torch
+    kind = ci.FFN_RELU_GATED if cfg.gated else ci.FFN_RELU
+    weights, acts = [], []
+    X = wl.prompt_hidden(cfg, device=device)
+    for l in range(cfg.L):
+        if cfg.planted:
+            w = wl.layer_weights(cfg, l, device=device)
+            A, _ = wl.planted_activations(cfg, l, cfg.T, device=device)
+        else:
+            w = wl.layer_weights(cfg, l, device=device)
+            A = torch.empty((cfg.T, cfg.d_ff), device=device)
+            Y = torch.empty((cfg.T, cfg.d_model), device=device)
+            ci.coreinfer_ffn_dense_ref(X, kind, w[0], w[1], w[2], None, None, A, Y)
+            V = X.float() + Y
+            X = (V / V.pow(2).mean(dim=1, keepdim=True).sqrt()).to(cfg.torch_dtype)
+        weights.append(w)
+        acts.append(A)
+    torch.cuda.synchronize()
+    return weights, acts
+
+
+def run_ours(args, cfg):
+    import torch
+    import torch.distributed as dist
+    import paper_2410_18311_b200 as ci
+    from paper_2410_18311_b200 import _build, workloads as wl
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        _build.build()
+    if world > 1:
+        dist.barrier()
+    ci.binding.load()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    weights, acts = prefill_inputs(ci, wl, cfg, dev)
+    stack = ci.pipeline.CoreSparseStack(cfg, device=dev)
+    steps_tok = cfg.decode_steps
+    xs = torch.cat([wl.decode_input(cfg, s, device=dev) for s in range(steps_tok)], dim=0)   # [steps, d]
+    ys = torch.empty((steps_tok, cfg.d_model), device=dev)
+    stream = torch.cuda.current_stream()
+
+    def request(ev=None):
+        if ev: ev[0].record(stream)
+        stack.prefill(acts, weights, stream)
+        if ev: ev[1].record(stream)
+        for s in range(steps_tok):
+            stack.decode(xs[s:s + 1], ys[s:s + 1], stream=stream)
+        if ev: ev[2].record(stream)
+
+    for _ in range(max(args.warmup, 3)):
+        request()
+    barrier()
+    stack.check()
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    barrier()
+    t_wall0 = time.perf_counter()
+    for i in range(args.steps):
+        request(evs[i])
+    barrier()
+    wall = time.perf_counter() - t_wall0
+    clocks = sampler.stop()
+    stack.check()
+    total_ms = evs[0][0].elapsed_time(evs[-1][2])
+    prefill_ms = sum(e[0].elapsed_time(e[1]) for e in evs) / args.steps
+    decode_ms = sum(e[1].elapsed_time(e[2]) for e in evs) / args.steps
+
+    total_ms_max = reduce_max(total_ms, dev)
+    value = whole_job_tokens_per_s(world, args.steps, steps_tok, total_ms_max)
+
+    # ---- per-stage latencies (outside the timed region) ----
+    def time_call(fn, reps=5):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        fn(); torch.cuda.synchronize()
+        a.record(stream)
+        for _ in range(reps): fn()
+        b.record(stream); torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+    sel_ms = time_call(lambda: [stack.select_layer(l, acts[l], None, stream) for l in range(cfg.L)]) / cfg.L
+    cmp_ms = time_call(lambda: [stack.compact_layer(l, *weights[l], stream=stream) for l in range(cfg.L)]) / cfg.L
+
+    # ---- end to end through the public API with host buffers ----
+    e2e = None
+    if not args.no_e2e:
+        acts_h = [torch.empty(a.shape, dtype=a.dtype, pin_memory=True).copy_(a) for a in acts]
+        xs_h = torch.empty(xs.shape, dtype=xs.dtype, pin_memory=True).copy_(xs)
+        ys_h = torch.empty(ys.shape, dtype=ys.dtype, pin_memory=True)
+        x_d = torch.empty((1, cfg.d_model), dtype=xs.dtype, device=dev)
+        y_d = torch.empty((1, cfg.d_model), device=dev)
+        acts_d = [torch.empty_like(a) for a in acts]
+
+        def request_e2e():
+            for l in range(cfg.L):
+                acts_d[l].copy_(acts_h[l], non_blocking=True)
+            stack.prefill(acts_d, weights, stream)
+            for s in range(steps_tok):
+                x_d.copy_(xs_h[s:s + 1], non_blocking=True)
+                stack.decode(x_d, y_d, stream=stream)
+                ys_h[s:s + 1].copy_(y_d, non_blocking=True)
+                stream.synchronize()          # the token's result is on the host before the next one starts
+        request_e2e()
+        barrier()
+        n_e2e = max(1, min(args.steps, 5))
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            request_e2e()
+        barrier()
+        dt = time.perf_counter() - t0
+        dt_max = reduce_max(dt, dev)
+        h2d = sum(a.numel() * 4 for a in acts) + steps_tok * cfg.d_model * cfg.esize
+        e2e = {"value": whole_job_tokens_per_s(world, n_e2e, steps_tok, dt_max * 1e3), "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": steps_tok * cfg.d_model * 4,
+               "requests_timed": n_e2e}
+        del acts_h, acts_d
+
+    # ---- the same kernel run dense (alpha = beta = 1), a few tokens ----
+    dense = None
+    if not args.no_dense and rank == 0:
+        try:
+            dcfg = cfg
+            dstack = ci.pipeline.CoreSparseStack(dcfg, device=dev, alpha=1.0, beta=1.0)
+            all_idx = torch.arange(cfg.d_ff, dtype=torch.int32, device=dev)
+            for l in range(cfg.L):
+                dstack.core_idx[l].copy_(all_idx)
+                dstack.compact_layer(l, *weights[l], stream=stream)
+            ntok = 8
+            ms = time_call(lambda: [dstack.decode(xs[s:s + 1], ys[s:s + 1], stream=stream) for s in range(ntok)], reps=2)
+            dstack.check()
+            dbytes = dstack.compacted_bytes_per_token()
+            dense = {"tok_s": ntok / (ms * 1e-3), "gbs": dbytes * ntok / (ms * 1e-3) / 1e9, "bytes_per_token": dbytes,
+                     "tokens_timed": 2 * ntok}
+            del dstack
+        except torch.OutOfMemoryError:
+            dense = {"skipped": "not enough free HBM for a second, dense copy of the stack"}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_src = measured_peak()
+    bytes_tok = stack.compacted_bytes_per_token() + cfg.L * 2 * cfg.d_model * 4
+    launch_s = decode_ms * 1e-3 / steps_tok
+    achieved = bytes_tok / launch_s / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": total_ms_max / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
+        "config": {"workload": cfg.name, "L": cfg.L, "d_model": cfg.d_model, "d_ff": cfg.d_ff, "T": cfg.T,
+                   "alpha": cfg.alpha, "beta": cfg.beta, "K": stack.K, "decode_steps": steps_tok, "batch": 1,
+                   "gated": cfg.gated, "step": "selection + compaction of all layers, then decode_steps tokens",
+                   "l2": "inputs larger than L2 (%.2f GB of compacted weights per token)" % (bytes_tok / 1e9),
+                   "parallelism": "independent requests per GPU, no collective"},
+        "decode": {"tok_s": steps_tok / (decode_ms * 1e-3), "ms_per_token": decode_ms / steps_tok,
+                   "gbs": achieved, "frac_of_8TBs": achieved / 8000.0},
+        "select_ms_per_layer": sel_ms, "compact_ms_per_layer": cmp_ms, "prefill_ms_per_request": prefill_ms,
+        "dense": dense,
+        "roofline": {"bound": "hbm", "kernel": "decode_stack_kernel", "achieved": achieved, "peak": peak,
+                     "unit": "GB/s", "frac": achieved / peak, "peak_source": "of " + peak_src,
+                     "bytes_per_launch": bytes_tok, "launch_us": launch_s * 1e6,
+                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH},
+        "e2e": e2e,
+        "gpu_launches": args.steps * (cfg.L * (stack.SELECT_KERNELS_PER_LAYER + stack.COMPACT_KERNELS_PER_LAYER)
+                                      + steps_tok * stack.DECODE_KERNELS_PER_TOKEN),
+        "clocks": clocks, "wall_s": wall,
+        "context": "paper (TITAN Xp, end to end, other workload): 10.33x over HuggingFace, 2.72x over PowerInfer",
+    }
+    if not args.no_cpu_baseline and world == 1:
+        line["cpu_baseline"] = oracle_sample(cfg, n_layers=2, n_tokens=4)
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    from paper_2410_18311_b200 import workloads as wl
+    cfg = wl.CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

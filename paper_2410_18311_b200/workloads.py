@@ -55,6 +55,8 @@ CONFIGS = {
     "relu-llama2-7b": Config(4, "relu-llama2-7b", "bf16", True, 32, 4096, 11008, 1024, 0.4, 0.25, 1, 256),
     "opt66b": Config(5, "opt66b", "bf16", False, 64, 9216, 36864, 512, 0.4, 0.2, 1, 128, planted=True),
 }
+# a seconds-scale stand-in with the same structure, for host-side tests of the harness
+CONFIGS["tiny"] = Config(9, "tiny", "bf16", False, 2, 256, 1024, 16, 0.4, 0.2, 1, 4)
 OPT13B_BETAS = (0.1, 0.2, 0.4, 1.0)
 OPT66B_TS = (128, 512, 2048, 4096)
 

@@ -1,0 +1,111 @@
+"""The whole path on the paper-shaped configurations: dense pre-fill activations -> selection
+-> compaction -> decode, each stage against the oracle on identical inputs."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2410_18311_b200 as ci
+from paper_2410_18311_b200 import workloads as wl
+from helpers import (require_gpu, gpu_select, gpu_compact, gpu_decode, to_f32_np, raw_np, assert_ffn_close)
+
+pytestmark = pytest.mark.gpu
+
+
+def _prefill_activations(cfg, layer, X):
+    w_up, w_gate, w_down = wl.layer_weights(cfg, layer, device="cuda")
+    H = torch.empty((X.shape[0], cfg.d_ff), device="cuda")
+    kind = ci.FFN_RELU_GATED if cfg.gated else ci.FFN_RELU
+    ci.coreinfer_ffn_dense_ref(X, kind, w_up, w_gate, w_down, None, None, H, None)
+    torch.cuda.synchronize()
+    return (w_up, w_gate, w_down), H, kind
+
+
+def test_config1_one_layer_fp32_full():
+    """One OPT-125M-shaped fp32 layer, T = 64, alpha 0.4, beta 0.2, 16 decode steps: every stage
+    compared in full."""
+    require_gpu()
+    cfg = wl.CONFIGS["opt125m-1layer"]
+    X = wl.prompt_hidden(cfg, device="cuda")
+    (w_up, w_gate, w_down), H, kind = _prefill_activations(cfg, 0, X)
+    H_o, _ = oracle.ffn_dense(to_f32_np(X), kind, to_f32_np(w_up), None, to_f32_np(w_down), want_y=False)
+    assert_ffn_close(H.cpu().numpy(), H_o, torch.float32)
+    S, f = gpu_select(H, cfg.alpha, cfg.beta)
+    S_o, f_o = oracle.select(H.cpu().numpy(), cfg.alpha, cfg.beta)      # same activation tensor
+    np.testing.assert_array_equal(f, f_o)
+    np.testing.assert_array_equal(S, S_o)
+    assert len(S) == 615
+    up_c, _, down_c, _ = gpu_compact(w_up, None, w_down, None, torch.from_numpy(S).cuda())
+    o_up, _, o_down, _ = oracle.compact(raw_np(w_up), None, raw_np(w_down), None, S_o)
+    assert raw_np(up_c).tobytes() == o_up.tobytes() and raw_np(down_c).tobytes() == o_down.tobytes()
+    for step in range(cfg.decode_steps):
+        x = wl.decode_input(cfg, step, device="cuda")
+        y = gpu_decode(x, kind, up_c, None, down_c)
+        y_o = oracle.ffn(to_f32_np(x), kind, o_up, None, o_down)
+        assert_ffn_close(y, y_o, torch.float32)
+
+
+def test_alpha_beta_one_reproduces_dense():
+    require_gpu()
+    cfg = wl.CONFIGS["opt125m-1layer"].with_(d_ff=1024, T=16)
+    X = wl.prompt_hidden(cfg, device="cuda")
+    (w_up, _, w_down), H, kind = _prefill_activations(cfg, 0, X)
+    S, _ = gpu_select(H, 1.0, 1.0)
+    np.testing.assert_array_equal(S, np.arange(cfg.d_ff))
+    up_c, _, down_c, _ = gpu_compact(w_up, None, w_down, None, torch.from_numpy(S).cuda())
+    x = wl.decode_input(cfg, 0, device="cuda")
+    y = gpu_decode(x, kind, up_c, None, down_c)
+    _, Y_o = oracle.ffn_dense(to_f32_np(x), kind, to_f32_np(w_up), None, to_f32_np(w_down), want_h=False)
+    assert_ffn_close(y, Y_o, torch.float32)
+
+
+@pytest.mark.parametrize("name,layers", [("opt6.7b", (0, 31)), ("opt13b", (7,)), ("relu-llama2-7b", (3,))])
+def test_bf16_configs_full_size_layers(name, layers):
+    """Full-size layers of the bf16 configurations (the set is bit-exact on the kernel's own
+    activations; activations, compaction and decode are checked on samples or in full)."""
+    require_gpu()
+    cfg = wl.CONFIGS[name]
+    X = wl.prompt_hidden(cfg, device="cuda")
+    rng = np.random.default_rng(0)
+    for layer in layers:
+        (w_up, w_gate, w_down), H, kind = _prefill_activations(cfg, layer, X)
+        # sampled rows of the activations against the oracle's own dense pass
+        rows = rng.choice(cfg.T, size=2, replace=False)
+        H_o, _ = oracle.ffn_dense(to_f32_np(X[rows]), kind, to_f32_np(w_up), to_f32_np(w_gate),
+                                  to_f32_np(w_down), want_y=False)
+        assert_ffn_close(H[rows].cpu().numpy(), H_o, torch.float32)
+        S, f = gpu_select(H, cfg.alpha, cfg.beta)
+        S_o, f_o = oracle.select(H.cpu().numpy(), cfg.alpha, cfg.beta)
+        np.testing.assert_array_equal(f, f_o)
+        np.testing.assert_array_equal(S, S_o)
+        assert len(S) == ci.coreinfer_count(cfg.beta, cfg.d_ff)
+        up_c, gate_c, down_c, _ = gpu_compact(w_up, w_gate, w_down, None, torch.from_numpy(S).cuda())
+        Sg = torch.from_numpy(S.astype(np.int64)).cuda()
+        assert torch.equal(up_c, w_up[Sg]) and torch.equal(down_c, w_down[:, Sg].t().contiguous())
+        o_up, o_gate, o_down, _ = oracle.compact(raw_np(w_up), raw_np(w_gate), raw_np(w_down), None, S_o)
+        assert raw_np(up_c).tobytes() == o_up.tobytes() and raw_np(down_c).tobytes() == o_down.tobytes()
+        if cfg.gated:
+            assert raw_np(gate_c).tobytes() == o_gate.tobytes()
+        for B in ((1, 8) if cfg.gated else (1,)):
+            x = wl.decode_input(cfg, layer, device="cuda", batch=B)
+            y = gpu_decode(x, kind, up_c, gate_c, down_c)
+            y_o = oracle.ffn(to_f32_np(x), kind, to_f32_np(up_c), to_f32_np(gate_c), to_f32_np(down_c))
+            assert_ffn_close(y, y_o, torch.bfloat16)
+
+
+@pytest.mark.parametrize("T", [128, 512])
+def test_opt66b_shaped_selection_and_decode(T):
+    require_gpu()
+    cfg = wl.CONFIGS["opt66b"]
+    A, core = wl.planted_activations(cfg, 0, T, device="cuda")
+    S, f = gpu_select(A, cfg.alpha, cfg.beta)
+    S_o, f_o = oracle.select(A.cpu().numpy(), cfg.alpha, cfg.beta)
+    np.testing.assert_array_equal(f, f_o)
+    np.testing.assert_array_equal(S, S_o)
+    assert len(S) == 7373 and np.isin(core.cpu().numpy(), S).all()
+    if T == 128:
+        up, _, down = wl.compacted_weights_random(cfg, 0, len(S), device="cuda")
+        x = wl.decode_input(cfg, 0, device="cuda")
+        y = gpu_decode(x, ci.FFN_RELU, up, None, down)
+        y_o = oracle.ffn(to_f32_np(x), ci.FFN_RELU, to_f32_np(up), None, to_f32_np(down))
+        assert_ffn_close(y, y_o, torch.bfloat16)
