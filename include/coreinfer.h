@@ -185,6 +185,37 @@ coreinfer_status coreinfer_ffn_decode_stack(const coreinfer_layer* layers, int32
                                             void* workspace, size_t workspace_bytes,
                                             void* cuda_stream);
 
+/* The same decode step as coreinfer_ffn_decode_stack for callers that cannot allocate device
+ * memory when they decode.  (The paper has no counterpart: this is a deployment convenience.)
+ * Typical cases: a server that gave all free HBM to its own pools at start-up and has nothing
+ * left to carve a workspace from; code running under a host framework that forbids cudaMalloc
+ * on its threads, since that call synchronises the device; a latency-critical loop that may
+ * not call an allocator.  The kernel's scratch (control words and per-layer reduction targets)
+ * sits in a fixed 4 MiB array inside the library image, so every GPU that loads the library
+ * gives up 4 MiB for the life of the process, and the call itself allocates nothing (no
+ * cudaMalloc / cudaFree, no allocating library routine).
+ *
+ * Arguments and results are those of coreinfer_ffn_decode_stack without the workspace pair.
+ * Limit: 256 + L * batch * d_model * 4 bytes must fit in 4 MiB (true for every shape up to
+ * 64 layers of d_model 9216); larger shapes return COREINFER_ERR_UNSUPPORTED and enqueue
+ * nothing -- use the workspace variant for them.
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress),
+ * which is set-up work rather than stream work: make that first call before starting any
+ * stream capture.
+ * All calls share the one array.  Each call clears the part it uses on `cuda_stream` before
+ * its kernel runs, so back-to-back calls on one stream are independent of what the previous
+ * one left behind; two calls that can overlap on the GPU (different streams, no ordering
+ * between them) race on it and give undefined results.  Because the array is private, the
+ * status word of a bounded wait that gave up cannot be read back after this entry point;
+ * callers that need that report use coreinfer_ffn_decode_stack.
+ * Errors: INVALID_ARG, UNSUPPORTED, CUDA. */
+coreinfer_status coreinfer_ffn_decode_stack_noalloc(const coreinfer_layer* layers, int32_t L,
+                                                    const void* x0, int32_t batch,
+                                                    coreinfer_dtype dtype, coreinfer_ffn_kind kind,
+                                                    int32_t d_model,
+                                                    float* y_last, float* y_layers, void* x_layers,
+                                                    void* cuda_stream);
+
 /* Synchronises `cuda_stream`, then reads the status word that the most recent
  * decode call using `workspace` left there: COREINFER_OK, or COREINFER_ERR_TIMEOUT
  * if a bounded device-side wait gave up (outputs of that call are then

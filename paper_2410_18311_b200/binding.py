@@ -26,6 +26,7 @@ SYMBOLS = (
     "coreinfer_compact",
     "coreinfer_ffn_decode_workspace_bytes", "coreinfer_ffn_decode",
     "coreinfer_ffn_decode_stack_workspace_bytes", "coreinfer_ffn_decode_stack",
+    "coreinfer_ffn_decode_stack_noalloc",
     "coreinfer_workspace_status",
     "coreinfer_ffn_dense_ref",
 )
@@ -82,6 +83,9 @@ def load() -> ctypes.CDLL:
     lib.coreinfer_ffn_decode_stack.restype = ctypes.c_int
     lib.coreinfer_ffn_decode_stack.argtypes = [ctypes.POINTER(Layer), i32, vp, i32, ctypes.c_int, ctypes.c_int,
                                                i32, vp, vp, vp, vp, sz, vp]
+    lib.coreinfer_ffn_decode_stack_noalloc.restype = ctypes.c_int
+    lib.coreinfer_ffn_decode_stack_noalloc.argtypes = [ctypes.POINTER(Layer), i32, vp, i32, ctypes.c_int,
+                                                       ctypes.c_int, i32, vp, vp, vp, vp]
     lib.coreinfer_workspace_status.restype = ctypes.c_int
     lib.coreinfer_workspace_status.argtypes = [vp, vp]
     lib.coreinfer_ffn_dense_ref.restype = ctypes.c_int
@@ -185,6 +189,17 @@ def coreinfer_ffn_decode_stack(layers, x0, kind, y_last, y_layers, x_layers, wor
     _check(load().coreinfer_ffn_decode_stack(layers, len(layers), _p(x0), batch, dtype_code(x0), int(kind),
                                              d_model, _p(y_last), _p(y_layers), _p(x_layers), _p(workspace),
                                              workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def coreinfer_ffn_decode_stack_noalloc(layers, x0, kind, y_last, y_layers, x_layers, stream=None):
+    """coreinfer_ffn_decode_stack for callers that cannot allocate: no workspace argument, the
+    scratch is a fixed 4 MiB array inside the library (shapes beyond it raise ERR_UNSUPPORTED).
+    Calls that may overlap on the GPU must not share it; make the first call on a device
+    outside stream capture."""
+    batch, d_model = x0.shape
+    _check(load().coreinfer_ffn_decode_stack_noalloc(layers, len(layers), _p(x0), batch, dtype_code(x0),
+                                                     int(kind), d_model, _p(y_last), _p(y_layers),
+                                                     _p(x_layers), _stream(stream)))
 
 
 def coreinfer_workspace_status(workspace, stream=None) -> None:

@@ -671,4 +671,66 @@ coreinfer_status coreinfer_ffn_decode_stack(const coreinfer_layer* layers, int32
                            workspace_bytes, need, (cudaStream_t)cuda_stream);
 }
 
+
+// ---------------------------------------------------------------------------
+// Variant of the stack entry point that needs no workspace from the caller.
+//
+// Some callers cannot obtain device memory at the time they decode: an inference server that
+// handed every free byte of HBM to its own pools at start-up, a plug-in that runs inside a host
+// framework which forbids cudaMalloc on its threads because the call synchronises the whole
+// device, a latency-critical loop in which an allocator call is not acceptable.  For them the
+// scratch of the stack kernel (control words + the per-layer reduction targets) lives in a
+// fixed array inside the library image.  The array costs kNoAllocScratchBytes of HBM on every
+// GPU that loads the library, for the life of the process.
+constexpr size_t kNoAllocScratchBytes = 4u << 20;   // 4 MiB: L * d_model * 4 + 256 must fit
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
+
+// The array's name is only a handle on the host; its device address comes from
+// cudaGetSymbolAddress, once per device, with that device current.
+static coreinfer_status noalloc_scratch_ptr(void** out)
+{
+    static thread_local void* cached[64] = {nullptr};
+    int dev = 0;
+    CI_CUDA(cudaGetDevice(&dev));
+    if (dev >= 0 && dev < 64 && cached[dev]) {
+        *out = cached[dev];
+        return COREINFER_OK;
+    }
+    void* p = nullptr;
+    CI_CUDA(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+    if (!p) CI_FAIL(COREINFER_ERR_CUDA, "cudaGetSymbolAddress returned a NULL address");
+    if (dev >= 0 && dev < 64) cached[dev] = p;
+    *out = p;
+    return COREINFER_OK;
+}
+
+coreinfer_status coreinfer_ffn_decode_stack_noalloc(const coreinfer_layer* layers, int32_t L,
+                                                    const void* x0, int32_t batch,
+                                                    coreinfer_dtype dtype, coreinfer_ffn_kind kind,
+                                                    int32_t d_model, float* y_last, float* y_layers,
+                                                    void* x_layers, void* cuda_stream)
+{
+    coreinfer_status s = check_common(x0, batch, dtype, kind, d_model);
+    if (s != COREINFER_OK) return s;
+    if (batch != 1) CI_FAIL(COREINFER_ERR_UNSUPPORTED, "the stack entry point is built for batch 1 (got %d)", batch);
+    if (!layers) CI_FAIL(COREINFER_ERR_INVALID_ARG, "layers is NULL");
+    if (L < 1 || L > COREINFER_MAX_LAYERS)
+        CI_FAIL(COREINFER_ERR_INVALID_ARG, "L = %d outside 1..%d", L, COREINFER_MAX_LAYERS);
+    if (!y_last || !aligned16(y_last)) CI_FAIL(COREINFER_ERR_INVALID_ARG, "y_last is NULL or not 16-byte aligned");
+    if ((y_layers && !aligned16(y_layers)) || (x_layers && !aligned16(x_layers)))
+        CI_FAIL(COREINFER_ERR_INVALID_ARG, "y_layers / x_layers not 16-byte aligned");
+    const size_t need = coreinfer_ffn_decode_stack_workspace_bytes(L, batch, d_model, 0);
+    if (need > kNoAllocScratchBytes)
+        CI_FAIL(COREINFER_ERR_UNSUPPORTED,
+                "L = %d, d_model = %d need %zu bytes of scratch; the built-in scratch holds %zu "
+                "(use coreinfer_ffn_decode_stack with a workspace)", L, d_model, need, kNoAllocScratchBytes);
+    void* scratch = nullptr;
+    s = noalloc_scratch_ptr(&scratch);
+    if (s != COREINFER_OK) return s;
+    // decode_stack_b1 zeroes the control words and the reduction targets it uses on the stream
+    // before the launch, so whatever the previous call left in the array does not matter.
+    return decode_stack_b1(layers, L, x0, dtype, kind, d_model, y_last, y_layers, x_layers, scratch,
+                           kNoAllocScratchBytes, need, (cudaStream_t)cuda_stream);
+}
+
 }  // extern "C"
