@@ -1,30 +1,37 @@
 // Decode-stage FFN over compacted core-neuron weights (Section 4.2), batch 1.
 //
-// One persistent kernel, one CTA per SM.  Per layer a CTA owns a contiguous slab
-// of the K core neurons and streams that slab's rows exactly once: first the up
-// (and gate) rows to form h for its neurons, then the matching rows of the
-// transposed down matrix to form its partial y.  Rows arrive through a ring of
-// shared-memory slots filled by 1-D bulk copies (one elected producer thread,
-// one mbarrier pair per slot).  The weights of a layer do not depend on its
-// input, so the producer runs ahead across layer boundaries and HBM stays busy
-// while the CTAs exchange partial outputs.
+// One persistent kernel, one CTA per SM.  Per layer a CTA owns a contiguous slab of the K core
+// neurons and streams that slab's rows exactly once: first the up (and gate) rows to form h for
+// its neurons, then the matching rows of the transposed down matrix to form its partial y.
+// Rows arrive through a ring of shared-memory slots filled by 1-D bulk copies (a producer warp,
+// one full/empty mbarrier pair per slot).  The weights of a layer do not depend on its input,
+// so the producer runs ahead across layer boundaries and HBM stays busy while the CTAs exchange
+// partial outputs.
 //
-// Exchange per layer: every CTA adds its partial y (d_model fp32) into one
-// global vector with vector reductions, then all CTAs meet at a grid barrier,
-// read the full y, and each forms the next layer's input redundantly in
-// registers.  Every wait (slot barriers, grid barrier) is bounded: when one
-// gives up, the CTA marks the workspace status word, stops waiting everywhere,
-// runs the rest of its schedule without synchronising on data, drains its own
-// copies in flight and returns.
+// Consumers own columns: thread t of a group holds the x values of its 16-byte vectors
+// t, t + 256, ... in registers for the whole layer and its partial y likewise.  They take ring
+// items in batches: wait for the batch, pull every vector of all its rows into registers with
+// no branch in between (so the loads overlap), free the slots at once, and only then do the
+// arithmetic; slots are held for a few hundred cycles whatever the arithmetic costs.  For rows
+// of at most 8 KB two such groups take alternate batches, so that one group's shared-memory
+// reads overlap the other's arithmetic; wider rows use one group.
+//
+// Exchange per layer: every group adds its partial y (d_model fp32) into a global vector with
+// vector reductions, then all CTAs meet at a grid barrier, read the full y, and every group
+// forms the next layer's input redundantly in registers.  Every wait (slot barriers, grid
+// barrier) is bounded: when one gives up, the CTA marks the workspace status word, stops
+// waiting everywhere, runs the rest of its schedule without synchronising on data, drains its
+// own copies in flight and returns.
 #include "common.cuh"
 
 namespace coreinfer {
 
 constexpr int kMaxSlots = 64;
-constexpr int kConsumerThreads = 256;
-constexpr int kConsumerWarps = kConsumerThreads / 32;
-constexpr int kBlockThreads = kConsumerThreads + 32;   // + one producer warp
+constexpr int kGroupThreads = 256;                     // consumer threads per group
+constexpr int kGroupWarps = kGroupThreads / 32;
 constexpr int kCtrlBytes = 256;                        // status word, barrier counter, padding
+constexpr int kYCopies = 2;                            // copies of a reduction target (spreads same-address adds)
+constexpr int kYBuffers = 3;                           // rotating targets: in use, being read, being cleared
 constexpr int kSplitRotate = 41;                       // per-layer rotation of the slab split
 constexpr long long kWaitCycles = 3000000000LL;        // bound of every device-side wait (~1.5 s)
 
@@ -44,16 +51,22 @@ struct DecodeParams {
     float* y_last;
     float* y_layers;
     void* x_layers;
-    float* ybuf;        // [L-1][d]: reduction targets of layers 0 .. L-2
+    float* ybuf;        // [kYBuffers][kYCopies][d]: reduction targets, buffer l % 3 serves layer l
     unsigned* ctrl;     // [0] status word, [1] grid-barrier arrival counter
     LayerDev layers[COREINFER_MAX_LAYERS];
 };
 
 __host__ __device__ __forceinline__ void slab_of(int cta, int G, int layer, int K, int* k0, int* k1)
 {
-    int vc = (int)(((long long)cta + (long long)layer * kSplitRotate) % G);
+    int vc = (cta + layer * kSplitRotate) % G;
     *k0 = (int)(((long long)vc * K) / G);
     *k1 = (int)(((long long)(vc + 1) * K) / G);
+}
+
+// items per consumer batch for one group (register budget: 4 * items * vectors per thread)
+__host__ __device__ constexpr int batch_for(int groups, int vpt)
+{
+    return groups == 2 ? 4 : (vpt <= 2 ? 8 : (vpt <= 4 ? 4 : 2));
 }
 
 // ------------------------------------------------------------ element types --
@@ -110,8 +123,8 @@ template <> struct Elem<float> {
 __device__ __forceinline__ bool wait_slot(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                           unsigned* status)
 {
-    if (*abort_flag) return false;
     if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
     const long long t0 = clock64();
     for (;;) {
         if (mbar_try_wait(bar, parity)) return true;
@@ -126,26 +139,29 @@ __device__ __forceinline__ bool wait_slot(uint32_t bar, uint32_t parity, volatil
 
 // All consumer threads call this.  The arrival counter is zeroed by the host before
 // the launch; barrier number b (0-based) completes when it reaches (b + 1) * G.
-__device__ __forceinline__ void grid_barrier(unsigned* ctrl, unsigned target,
-                                             volatile int* abort_flag)
+__device__ __forceinline__ void grid_barrier(unsigned* ctrl, unsigned target, volatile int* abort_flag,
+                                             int nthreads)
 {
-    named_bar_sync(1, kConsumerThreads);
+    named_bar_sync(1, nthreads);
     if (threadIdx.x == 0 && !*abort_flag) {
         __threadfence();
         atomicAdd(&ctrl[1], 1u);
         const long long t0 = clock64();
+        unsigned it = 0;
         for (;;) {
             if (ld_acquire_gpu(&ctrl[1]) >= target) break;
-            if (ld_acquire_gpu(&ctrl[0]) != kStatusOk) { *abort_flag = 1; break; }
-            if (clock64() - t0 > kWaitCycles) {
-                *abort_flag = 1;
-                atomicMax(&ctrl[0], (unsigned)kStatusTimeout);
-                break;
+            if ((++it & 255u) == 0u) {             // now and then: has another CTA given up? out of time?
+                if (ld_acquire_gpu(&ctrl[0]) != kStatusOk) { *abort_flag = 1; break; }
+                if (clock64() - t0 > kWaitCycles) {
+                    *abort_flag = 1;
+                    atomicMax(&ctrl[0], (unsigned)kStatusTimeout);
+                    break;
+                }
             }
         }
         __threadfence();
     }
-    named_bar_sync(1, kConsumerThreads);
+    named_bar_sync(1, nthreads);
 }
 
 // 8 values per lane -> 8 warp totals, one per group of 4 lanes (9 shuffles).
@@ -178,27 +194,30 @@ __device__ __forceinline__ float warp_reduce8(const float (&v)[8], int lane)
 }
 
 // ------------------------------------------------------------------- kernel --
-// Ring stream order of one CTA and one layer (producer and consumers walk it in
-// lock step): for each group of rows {g0 .. g0+R-1}: the up rows, then (gated)
-// the gate rows; after all groups, the down rows k0 .. k1-1.
-template <typename T, int VPT, bool GATED>
-__global__ void __launch_bounds__(kBlockThreads, 1)
+// Ring stream order of one CTA and one layer (producer and consumers walk it in lock step): for
+// each slab row k0 .. k1-1 its up row, then (gated) its gate row; after those, the down rows
+// k0 .. k1-1.  Within each of the two phases the items are cut into batches of BATCH; batch b
+// belongs to consumer group b % NG.
+template <typename T, int NG, int VPT, bool GATED>
+__global__ void __launch_bounds__(NG * kGroupThreads + 32, 1)
 decode_stack_kernel(const __grid_constant__ DecodeParams p)
 {
     using E = Elem<T>;
     constexpr int PAIRS = E::kPairs;
-    constexpr int EPV = PAIRS * 2;               // elements per 16-byte vector
-    constexpr int R = GATED ? 4 : 8;             // rows per up-phase group
+    constexpr int EPV = PAIRS * 2;                   // elements per 16-byte vector
     constexpr int NMAT = GATED ? 2 : 1;
+    constexpr int NC = NG * kGroupThreads;           // consumer threads
+    constexpr int BATCH = batch_for(NG, VPT);        // ring items per batch
+    constexpr int FLUSH = 8 / BATCH;                 // own up batches per cross-lane reduction
 
     extern __shared__ __align__(128) uint8_t smem[];
     uint8_t* ring = smem;
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(ring + (size_t)p.n_slots * p.slot_bytes);
     uint64_t* empty_bar = full_bar + kMaxSlots;
-    float* red = reinterpret_cast<float*>(empty_bar + kMaxSlots);   // [NMAT][warps][rmax]
-    float* h_s = red + NMAT * kConsumerWarps * p.rmax;              // [rmax]
-    float* ss_red = h_s + p.rmax;                                   // [warps]
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(ss_red + kConsumerWarps);
+    float* red = reinterpret_cast<float*>(empty_bar + kMaxSlots);   // [NMAT][kGroupWarps][rmax]
+    float* h_s = red + NMAT * kGroupWarps * p.rmax;                 // [rmax]
+    float* ss_red = h_s + p.rmax;                                   // [NG][kGroupWarps]
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(ss_red + NG * kGroupWarps);
 
     const int tid = threadIdx.x;
     const int G = gridDim.x;
@@ -208,7 +227,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) {
             mbar_init(smem_u32(&full_bar[s]), 1);
-            mbar_init(smem_u32(&empty_bar[s]), kConsumerWarps);
+            mbar_init(smem_u32(&empty_bar[s]), kGroupWarps);     // the warps of the group that reads the slot
         }
         *abort_flag = 0;
         mbar_fence_init();
@@ -216,83 +235,131 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
     __syncthreads();
 
     // ======================================================== producer warp ==
-    if (tid >= kConsumerThreads) {
-        if (tid == kConsumerThreads) {
-            long long it = 0;
-            bool live = true;
-            auto issue = [&](const uint8_t* src) {
-                const int slot = (int)(it % NS);
-                const uint32_t ph = (uint32_t)((it / NS) & 1);
-                if (live && !wait_slot(smem_u32(&empty_bar[slot]), ph ^ 1u, abort_flag, p.ctrl))
-                    live = false;
-                if (live) {
-                    const uint32_t fb = smem_u32(&full_bar[slot]);
-                    mbar_arrive_expect_tx(fb, (uint32_t)p.row_bytes);
-                    bulk_g2s(smem_u32(ring + (size_t)slot * p.slot_bytes), src, (uint32_t)p.row_bytes, fb);
-                    ++it;
+    // Up to eight lanes issue copies: one round fills up to min(8, ring slots) consecutive ring
+    // items, lane j taking item j of the round (its own slot, its own wait on that slot's
+    // "empty" barrier), so the latency of one issue is not the issue rate.
+    if (tid >= NC) {
+        const int lane = tid - NC;
+        const int round_max = NS < 8 ? NS : 8;
+        int slot0 = 0;                // ring position of the round's first item
+        uint32_t phase0 = 0;          // parity of the ring pass that position belongs to
+        long long issued = 0;
+        for (int l = 0; l < p.L; ++l) {
+            const LayerDev& ly = p.layers[l];
+            int k0, k1;
+            slab_of(cta, G, l, ly.K, &k0, &k1);
+            const int n = k1 - k0;
+            const int n_up = n * NMAT;            // items of the up (+ gate) phase
+            const int total = n_up + n;           // + the down rows
+            for (int q0 = 0; q0 < total; q0 += round_max) {
+                if (*abort_flag) break;
+                const int cnt = min(round_max, total - q0);
+                if (lane < cnt) {
+                    const int q = q0 + lane;
+                    const uint8_t* src;
+                    if (q < n_up) {
+                        const int row = k0 + q / NMAT;
+                        src = ((GATED && (q % NMAT)) ? ly.gate : ly.up) + (size_t)row * p.row_bytes;
+                    } else {
+                        src = ly.down + (size_t)(k0 + q - n_up) * p.row_bytes;
+                    }
+                    int sl = slot0 + lane;
+                    uint32_t ph = phase0;
+                    if (sl >= NS) { sl -= NS; ph ^= 1u; }
+                    if (wait_slot(smem_u32(&empty_bar[sl]), ph ^ 1u, abort_flag, p.ctrl)) {
+                        const uint32_t fb = smem_u32(&full_bar[sl]);
+                        mbar_arrive_expect_tx(fb, (uint32_t)p.row_bytes);
+                        bulk_g2s(smem_u32(ring + (size_t)sl * p.slot_bytes), src, (uint32_t)p.row_bytes, fb);
+                    }
                 }
-            };
-            for (int l = 0; l < p.L && live; ++l) {
-                const LayerDev& ly = p.layers[l];
-                int k0, k1;
-                slab_of(cta, G, l, ly.K, &k0, &k1);
-                for (int g0 = k0; g0 < k1 && live; g0 += R) {
-                    const int ge = min(g0 + R, k1);
-                    for (int k = g0; k < ge; ++k) issue(ly.up + (size_t)k * p.row_bytes);
-                    if (GATED)
-                        for (int k = g0; k < ge; ++k) issue(ly.gate + (size_t)k * p.row_bytes);
-                }
-                for (int k = k0; k < k1 && live; ++k) issue(ly.down + (size_t)k * p.row_bytes);
+                __syncwarp();
+                slot0 += cnt;
+                if (slot0 >= NS) { slot0 -= NS; phase0 ^= 1u; }
+                issued += cnt;
             }
-            // Do not leave while a copy into this CTA's shared memory is in flight.
-            const long long first = it > NS ? it - NS : 0;
-            for (long long i = first; i < it; ++i) {
-                const uint32_t fb = smem_u32(&full_bar[(int)(i % NS)]);
-                const uint32_t ph = (uint32_t)((i / NS) & 1);
-                const long long t0 = clock64();
-                while (!mbar_try_wait(fb, ph))
-                    if (clock64() - t0 > kWaitCycles) { atomicMax(p.ctrl, (unsigned)kStatusTimeout); break; }
-            }
+        }
+        // Do not leave while a copy into this CTA's shared memory is in flight: wait (bounded)
+        // for the last copy issued into every slot.  (After an abort a counted item may not have
+        // been issued; its wait then runs into the bound, which only delays the return.)
+        for (int sl = lane; sl < NS; sl += 32) {
+            const long long uses = issued / NS + (sl < (int)(issued % NS) ? 1 : 0);
+            if (uses == 0) continue;
+            const uint32_t fb = smem_u32(&full_bar[sl]);
+            const uint32_t ph = (uint32_t)((uses - 1) & 1);
+            const long long t0 = clock64();
+            while (!mbar_try_wait(fb, ph))
+                if (clock64() - t0 > kWaitCycles) { atomicMax(p.ctrl, (unsigned)kStatusTimeout); break; }
         }
         return;
     }
 
     // ============================================================ consumers ==
+    const int grp = tid / kGroupThreads;          // consumer group of this thread
+    const int gt = tid % kGroupThreads;           // thread within the group
     const int lane = tid & 31;
-    const int warp = tid >> 5;
+    const int gw = gt >> 5;                       // warp within the group
     const int nv = p.nv;
     const int d = p.d;
 
-    // this thread's columns: 16-byte vectors tid, tid + 256, ...
+    // this thread's columns: 16-byte vectors gt, gt + 256, ...  vofs[] is clamped so that loads
+    // never need a branch (threads beyond the row read vector 0 against a zero x).
     float2 xr[VPT][PAIRS];
+    int vofs[VPT];
 #pragma unroll
     for (int i = 0; i < VPT; ++i) {
-        const int v = tid + i * kConsumerThreads;
+        const int v = gt + i * kGroupThreads;
+        vofs[i] = (v < nv ? v : 0) * 16;
         uint4 q = make_uint4(0, 0, 0, 0);
         if (v < nv) q = reinterpret_cast<const uint4*>(p.x0)[v];
         E::unpack(q, xr[i]);
-        if (p.x_layers && cta == 0 && v < nv) reinterpret_cast<uint4*>(p.x_layers)[v] = q;
-    }
-    if (p.L > 1) {   // reductions of the last layer land here after at least one grid barrier
-        const uint4 z = make_uint4(0, 0, 0, 0);
-        if (cta == 0)
-            for (int i = tid; i < d / 4; i += kConsumerThreads) reinterpret_cast<uint4*>(p.y_last)[i] = z;
-        if (p.y_layers && cta == 1 % G)
-            for (int i = tid; i < d / 4; i += kConsumerThreads)
-                reinterpret_cast<uint4*>(p.y_layers + (size_t)(p.L - 1) * d)[i] = z;
+        if (p.x_layers && cta == 0 && grp == 0 && v < nv) reinterpret_cast<uint4*>(p.x_layers)[v] = q;
     }
 
-    long long it = 0;
-    auto acquire = [&]() -> const uint8_t* {
-        const int slot = (int)(it % NS);
-        wait_slot(smem_u32(&full_bar[slot]), (uint32_t)((it / NS) & 1), abort_flag, p.ctrl);
-        return ring + (size_t)slot * p.slot_bytes;
+    int slot = 0;                 // ring position of the next item of the stream
+    uint32_t phase = 0;
+    auto skip_n = [&](int n) {    // items that belong to the other group
+        slot += n;
+        if (slot >= NS) { slot -= NS; phase ^= 1u; }
     };
-    auto release = [&]() {
-        const int slot = (int)(it % NS);
+    // wait for the next n items, pull them into registers (q[j][i] = vector i of item j), free them
+    auto fetch = [&](uint4 (&q)[BATCH][VPT], int n) {
+        {
+            int sl = slot;
+            uint32_t ph = phase;
+            for (int j = 0; j < n; ++j) {
+                wait_slot(smem_u32(&full_bar[sl]), ph, abort_flag, p.ctrl);
+                if (++sl == NS) { sl = 0; ph ^= 1u; }
+            }
+        }
+        if (n == BATCH) {
+#pragma unroll
+            for (int j = 0; j < BATCH; ++j) {
+                int sl = slot + j;
+                if (sl >= NS) sl -= NS;
+                const uint8_t* row = ring + (size_t)sl * p.slot_bytes;
+#pragma unroll
+                for (int i = 0; i < VPT; ++i) q[j][i] = *reinterpret_cast<const uint4*>(row + vofs[i]);
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < BATCH; ++j) {
+                int sl = slot + (j < n ? j : 0);
+                if (sl >= NS) sl -= NS;
+                const uint8_t* row = ring + (size_t)sl * p.slot_bytes;
+#pragma unroll
+                for (int i = 0; i < VPT; ++i) {
+                    q[j][i] = *reinterpret_cast<const uint4*>(row + vofs[i]);
+                    if (j >= n) q[j][i] = make_uint4(0, 0, 0, 0);
+                }
+            }
+        }
         __syncwarp();
-        if (lane == 0 && !*abort_flag) mbar_arrive(smem_u32(&empty_bar[slot]));
-        ++it;
+        if (lane < n && !*abort_flag) {
+            int sl = slot + lane;
+            if (sl >= NS) sl -= NS;
+            mbar_arrive(smem_u32(&empty_bar[sl]));
+        }
+        skip_n(n);
     };
 
     for (int l = 0; l < p.L; ++l) {
@@ -300,53 +367,66 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
         int k0, k1;
         slab_of(cta, G, l, ly.K, &k0, &k1);
         const int nrows = k1 - k0;
+        const int n_up = nrows * NMAT;
 
         // ------------------------------------------------ up (+ gate) phase --
-        for (int g0 = k0; g0 < k1; g0 += R) {
-            const int ge = min(g0 + R, k1);
+        {
+            const int nb = (n_up + BATCH - 1) / BATCH;
             float part[8];
 #pragma unroll
             for (int j = 0; j < 8; ++j) part[j] = 0.f;
+            int own = 0;                          // own batches accumulated in part[]
+            int first_b = 0;                      // first of them
+            for (int b = 0; b < nb; ++b) {
+                const int cnt = min(BATCH, n_up - b * BATCH);
+                if (NG > 1 && (b % NG) != grp) { skip_n(cnt); continue; }
+                uint4 q[BATCH][VPT];
+                fetch(q, cnt);
+                if (own == 0) first_b = b;
 #pragma unroll
-            for (int m = 0; m < NMAT; ++m) {
+                for (int f = 0; f < FLUSH; ++f) {
+                    if (f == own) {               // uniform; keeps part[] statically indexed
 #pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    if (g0 + r < ge) {
-                        const uint8_t* row = acquire();
-                        float2 acc = make_float2(0.f, 0.f);
+                        for (int j = 0; j < BATCH; ++j) {
+                            float2 acc = make_float2(0.f, 0.f);
 #pragma unroll
-                        for (int i = 0; i < VPT; ++i) {
-                            const int v = tid + i * kConsumerThreads;
-                            if (v < nv) {
-                                const uint4 q = *reinterpret_cast<const uint4*>(row + (size_t)v * 16);
+                            for (int i = 0; i < VPT; ++i) {
                                 float2 w[PAIRS];
-                                E::unpack(q, w);
+                                E::unpack(q[j][i], w);
 #pragma unroll
                                 for (int c = 0; c < PAIRS; ++c) acc = __ffma2_rn(w[c], xr[i][c], acc);
                             }
+                            part[f * BATCH + j] = acc.x + acc.y;
                         }
-                        release();
-                        part[m * R + r] = acc.x + acc.y;
                     }
                 }
-            }
-            const float tot = warp_reduce8(part, lane);
-            if ((lane & 3) == 0) {
-                const int j = ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);
-                const int m = j / R, r = j % R;
-                if (g0 + r < ge) red[(m * kConsumerWarps + warp) * p.rmax + (g0 - k0) + r] = tot;
+                ++own;
+                const bool flush = own == FLUSH || b + NG >= nb;
+                if (flush) {
+                    const float tot = warp_reduce8(part, lane);
+                    if ((lane & 3) == 0) {
+                        const int vi = ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);
+                        const int f = vi / BATCH, j = vi % BATCH;          // own batch f of the window, item j
+                        const int item = (first_b + f * NG) * BATCH + j;   // position in the up phase
+                        if (f < own && item < n_up)
+                            red[((item % NMAT) * kGroupWarps + gw) * p.rmax + item / NMAT] = tot;
+                    }
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) part[j] = 0.f;
+                    own = 0;
+                }
             }
         }
-        named_bar_sync(1, kConsumerThreads);
-        for (int r = tid; r < nrows; r += kConsumerThreads) {
+        named_bar_sync(1, NC);
+        for (int r = tid; r < nrows; r += NC) {
             float u = 0.f;
 #pragma unroll
-            for (int w = 0; w < kConsumerWarps; ++w) u += red[w * p.rmax + r];
+            for (int w = 0; w < kGroupWarps; ++w) u += red[w * p.rmax + r];
             float h;
             if (GATED) {
                 float g = 0.f;
 #pragma unroll
-                for (int w = 0; w < kConsumerWarps; ++w) g += red[(kConsumerWarps + w) * p.rmax + r];
+                for (int w = 0; w < kGroupWarps; ++w) g += red[(kGroupWarps + w) * p.rmax + r];
                 h = fmaxf(g, 0.f) * u;
             } else {
                 if (ly.bup) u += E::load1(ly.bup, k0 + r);
@@ -354,74 +434,92 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
             }
             h_s[r] = h;
         }
-        named_bar_sync(1, kConsumerThreads);
+        named_bar_sync(1, NC);
 
         // ------------------------------------------------------- down phase --
         float2 yacc[VPT][PAIRS];
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
-            const int v = tid + i * kConsumerThreads;
+            const int v = gt + i * kGroupThreads;
 #pragma unroll
             for (int c = 0; c < PAIRS; ++c) yacc[i][c] = make_float2(0.f, 0.f);
-            if (cta == 0 && ly.bdown && v < nv) {   // the bias enters the sum exactly once
+            if (cta == 0 && grp == 0 && ly.bdown && v < nv) {   // the bias enters the sum exactly once
 #pragma unroll
                 for (int c = 0; c < PAIRS; ++c)
                     yacc[i][c] = make_float2(E::load1(ly.bdown, v * EPV + 2 * c),
                                              E::load1(ly.bdown, v * EPV + 2 * c + 1));
             }
         }
-        for (int r = 0; r < nrows; ++r) {
-            const uint8_t* row = acquire();
-            const float hk = h_s[r];
-            if (hk != 0.f) {
-                const float2 hh = make_float2(hk, hk);
+        {
+            const int nb = (nrows + BATCH - 1) / BATCH;
+            for (int b = 0; b < nb; ++b) {
+                const int cnt = min(BATCH, nrows - b * BATCH);
+                if (NG > 1 && (b % NG) != grp) { skip_n(cnt); continue; }
+                uint4 q[BATCH][VPT];
+                fetch(q, cnt);
 #pragma unroll
-                for (int i = 0; i < VPT; ++i) {
-                    const int v = tid + i * kConsumerThreads;
-                    if (v < nv) {
-                        const uint4 q = *reinterpret_cast<const uint4*>(row + (size_t)v * 16);
-                        float2 w[PAIRS];
-                        E::unpack(q, w);
+                for (int j = 0; j < BATCH; ++j) {
+                    const float hk = (j < cnt) ? h_s[b * BATCH + j] : 0.f;
+                    if (hk != 0.f) {                              // uniform: ReLU zeros cost no arithmetic
+                        const float2 hh = make_float2(hk, hk);
 #pragma unroll
-                        for (int c = 0; c < PAIRS; ++c) yacc[i][c] = __ffma2_rn(w[c], hh, yacc[i][c]);
+                        for (int i = 0; i < VPT; ++i) {
+                            float2 w[PAIRS];
+                            E::unpack(q[j][i], w);
+#pragma unroll
+                            for (int c = 0; c < PAIRS; ++c) yacc[i][c] = __ffma2_rn(w[c], hh, yacc[i][c]);
+                        }
                     }
                 }
             }
-            release();
         }
 
         // ----------------------------------------- cross-CTA sum of partial y --
+        // Every group adds its partial into one of kYCopies copies of the layer's target (adds to
+        // one address are serialised in L2, so they are spread); after the grid barrier every
+        // thread sums the copies for its columns.  Targets rotate over three buffers: while layer
+        // l's is read, the one layer l+2 will use is cleared (last read before the barrier of l).
         const bool last = (l == p.L - 1);
-        float* ytarget = last ? p.y_last : p.ybuf + (size_t)l * d;
+        float* ybase = p.ybuf + (size_t)(l % kYBuffers) * kYCopies * d;
+        float* ytarget = ybase + (size_t)((cta + grp) & (kYCopies - 1)) * d;
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
-            const int v = tid + i * kConsumerThreads;
+            const int v = gt + i * kGroupThreads;
             if (v < nv) {
 #pragma unroll
-                for (int c = 0; c < PAIRS; c += 2) {
-                    float* dst = ytarget + (size_t)v * EPV + 2 * c;
-                    red_add_v4(dst, yacc[i][c].x, yacc[i][c].y, yacc[i][c + 1].x, yacc[i][c + 1].y);
-                    if (last && p.y_layers)
-                        red_add_v4(p.y_layers + (size_t)l * d + (size_t)v * EPV + 2 * c, yacc[i][c].x,
-                                   yacc[i][c].y, yacc[i][c + 1].x, yacc[i][c + 1].y);
-                }
+                for (int c = 0; c < PAIRS; c += 2)
+                    red_add_v4(ytarget + (size_t)v * EPV + 2 * c, yacc[i][c].x, yacc[i][c].y, yacc[i][c + 1].x,
+                               yacc[i][c + 1].y);
             }
         }
-        if (last) break;
 
-        grid_barrier(p.ctrl, (unsigned)(l + 1) * (unsigned)G, abort_flag);
+        grid_barrier(p.ctrl, (unsigned)(l + 1) * (unsigned)G, abort_flag, NC);
+
+        {
+            float4* z = reinterpret_cast<float4*>(p.ybuf + (size_t)((l + 2) % kYBuffers) * kYCopies * d);
+            const int n4 = kYCopies * d / 4;
+            for (int i = cta * NC + tid; i < n4; i += G * NC) z[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
 
         // ------------------------- next input: (x + y) / rms(x + y), rounded --
         float ss = 0.f;
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
-            const int v = tid + i * kConsumerThreads;
+            const int v = gt + i * kGroupThreads;
             if (v < nv) {
 #pragma unroll
                 for (int c = 0; c < PAIRS; c += 2) {
-                    const float4 t = __ldcg(reinterpret_cast<const float4*>(ytarget + (size_t)v * EPV + 2 * c));
-                    if (p.y_layers && cta == l % G)
-                        *reinterpret_cast<float4*>(p.y_layers + (size_t)l * d + (size_t)v * EPV + 2 * c) = t;
+                    float4 u[kYCopies];
+#pragma unroll
+                    for (int cp = 0; cp < kYCopies; ++cp)
+                        u[cp] = __ldcg(reinterpret_cast<const float4*>(ybase + (size_t)cp * d + (size_t)v * EPV + 2 * c));
+                    float4 t = u[0];
+#pragma unroll
+                    for (int cp = 1; cp < kYCopies; ++cp) { t.x += u[cp].x; t.y += u[cp].y; t.z += u[cp].z; t.w += u[cp].w; }
+                    if (cta == l % G && grp == 0) {
+                        if (p.y_layers) *reinterpret_cast<float4*>(p.y_layers + (size_t)l * d + (size_t)v * EPV + 2 * c) = t;
+                        if (last) *reinterpret_cast<float4*>(p.y_last + (size_t)v * EPV + 2 * c) = t;
+                    }
                     xr[i][c].x += t.x;
                     xr[i][c].y += t.y;
                     xr[i][c + 1].x += t.z;
@@ -434,23 +532,25 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
                 }
             }
         }
+        if (last) break;
+        // every group holds all columns, so each forms the norm on its own (same sums, same order)
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-        if (lane == 0) ss_red[warp] = ss;
-        named_bar_sync(1, kConsumerThreads);
+        if (lane == 0) ss_red[grp * kGroupWarps + gw] = ss;
+        named_bar_sync(2 + grp, kGroupThreads);
         float tot = 0.f;
 #pragma unroll
-        for (int w = 0; w < kConsumerWarps; ++w) tot += ss_red[w];
+        for (int w = 0; w < kGroupWarps; ++w) tot += ss_red[grp * kGroupWarps + w];
         const float inv = 1.0f / sqrtf(tot / (float)d);
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
-            const int v = tid + i * kConsumerThreads;
+            const int v = gt + i * kGroupThreads;
 #pragma unroll
             for (int c = 0; c < PAIRS; ++c) {
                 xr[i][c].x = E::round(xr[i][c].x * inv);
                 xr[i][c].y = E::round(xr[i][c].y * inv);
             }
-            if (p.x_layers && cta == (l + 1) % G && v < nv)
+            if (p.x_layers && cta == (l + 1) % G && grp == 0 && v < nv)
                 reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(p.x_layers) +
                                          (size_t)(l + 1) * p.row_bytes)[v] = E::pack(xr[i]);
         }
@@ -458,20 +558,19 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
 }
 
 // ------------------------------------------------------------------- host ---
-static size_t fixed_smem_bytes(int rmax, bool gated)
+static size_t fixed_smem_bytes(int rmax, bool gated, int groups)
 {
     size_t b = 2 * kMaxSlots * sizeof(uint64_t);
-    b += (size_t)(gated ? 2 : 1) * kConsumerWarps * rmax * sizeof(float);
+    b += (size_t)(gated ? 2 : 1) * kGroupWarps * rmax * sizeof(float);
     b += (size_t)rmax * sizeof(float);
-    b += kConsumerWarps * sizeof(float) + 16;
+    b += (size_t)groups * kGroupWarps * sizeof(float) + 16;
     return (b + 127) & ~(size_t)127;
 }
 
-template <typename T, int VPT, bool GATED>
-static coreinfer_status launch_one(const DecodeParams& p, int grid, size_t smem, bool cooperative,
-                                   cudaStream_t st)
+template <typename T, int NG, int VPT, bool GATED>
+static coreinfer_status launch_one(const DecodeParams& p, int grid, size_t smem, cudaStream_t st)
 {
-    auto kern = decode_stack_kernel<T, VPT, GATED>;
+    auto kern = decode_stack_kernel<T, NG, VPT, GATED>;
     static thread_local size_t configured[64] = {0};
     int dev = 0;
     CI_CUDA(cudaGetDevice(&dev));
@@ -481,27 +580,36 @@ static coreinfer_status launch_one(const DecodeParams& p, int grid, size_t smem,
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3(kBlockThreads);
+    cfg.blockDim = dim3((unsigned)(NG * kGroupThreads + 32));
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeCooperative;
-    attr[0].val.cooperative = cooperative ? 1 : 0;
+    attr[0].id = cudaLaunchAttributeCooperative;    // the CTAs wait on one another at layer ends
+    attr[0].val.cooperative = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     CI_CUDA(cudaLaunchKernelEx(&cfg, kern, p));
     return COREINFER_OK;
 }
 
-template <typename T, bool GATED>
-static coreinfer_status launch_vpt(int vpt, const DecodeParams& p, int grid, size_t smem, bool coop,
-                                   cudaStream_t st)
+static int groups_for(int nv) { return nv <= 2 * kGroupThreads ? 2 : 1; }
+static int vpt_for(int nv)
 {
-    if (vpt <= 1) return launch_one<T, 1, GATED>(p, grid, smem, coop, st);
-    if (vpt <= 2) return launch_one<T, 2, GATED>(p, grid, smem, coop, st);
-    if (vpt <= 3) return launch_one<T, 3, GATED>(p, grid, smem, coop, st);
-    if (vpt <= 5) return launch_one<T, 5, GATED>(p, grid, smem, coop, st);
-    return launch_one<T, 8, GATED>(p, grid, smem, coop, st);
+    const int v = (nv + kGroupThreads - 1) / kGroupThreads;
+    return v <= 1 ? 1 : v <= 2 ? 2 : v <= 3 ? 3 : v <= 5 ? 5 : 8;
+}
+
+template <typename T, bool GATED>
+static coreinfer_status launch_shape(int groups, int vpt, const DecodeParams& p, int grid, size_t smem,
+                                     cudaStream_t st)
+{
+    if (groups == 2) {
+        if (vpt <= 1) return launch_one<T, 2, 1, GATED>(p, grid, smem, st);
+        return launch_one<T, 2, 2, GATED>(p, grid, smem, st);
+    }
+    if (vpt <= 3) return launch_one<T, 1, 3, GATED>(p, grid, smem, st);
+    if (vpt <= 5) return launch_one<T, 1, 5, GATED>(p, grid, smem, st);
+    return launch_one<T, 1, 8, GATED>(p, grid, smem, st);
 }
 
 static coreinfer_status check_common(const void* x, int batch, coreinfer_dtype dtype,
@@ -530,6 +638,11 @@ static coreinfer_status check_layer(const coreinfer_layer& ly, int l, coreinfer_
     if (!gated && ly.w_gate_c) CI_FAIL(COREINFER_ERR_INVALID_ARG, "layer %d: w_gate_c given for a non-gated FFN", l);
     if (gated && ly.b_up_c) CI_FAIL(COREINFER_ERR_INVALID_ARG, "layer %d: the gated FFN has no up bias", l);
     return COREINFER_OK;
+}
+
+static size_t b1_workspace_bytes(int d_model)
+{
+    return kCtrlBytes + (size_t)kYBuffers * kYCopies * (size_t)d_model * sizeof(float);
 }
 
 // Shared by the one-layer and the stack entry points (batch 1).
@@ -569,12 +682,14 @@ static coreinfer_status decode_stack_b1(const coreinfer_layer* layers, int L, co
         if (layers[l].K > Kmax) Kmax = layers[l].K;
     }
     p.rmax = (Kmax + G - 1) / G + 1;
-    const int vpt = (p.nv + kConsumerThreads - 1) / kConsumerThreads;
-    if (vpt > 8)
+    const int groups = groups_for(p.nv);
+    if ((p.nv + kGroupThreads - 1) / kGroupThreads > 8)
         CI_FAIL(COREINFER_ERR_UNSUPPORTED, "d_model %d is too wide for this kernel (max %d bytes per row)",
-                d_model, 8 * kConsumerThreads * 16);
-    const size_t fixed = fixed_smem_bytes(p.rmax, gated);
-    if (fixed + (size_t)p.slot_bytes > (size_t)di.smem_optin)
+                d_model, 8 * kGroupThreads * 16);
+    const int vpt = groups == 2 ? ((p.nv + kGroupThreads - 1) / kGroupThreads <= 1 ? 1 : 2) : vpt_for(p.nv);
+    const int batch = batch_for(groups, groups == 2 ? vpt : (vpt <= 3 ? 3 : vpt));
+    const size_t fixed = fixed_smem_bytes(p.rmax, gated, groups);
+    if (fixed + (size_t)batch * p.slot_bytes > (size_t)di.smem_optin)
         CI_FAIL(COREINFER_ERR_UNSUPPORTED, "K = %d, d_model = %d do not fit in shared memory", Kmax, d_model);
     long long slots = ((long long)di.smem_optin - (long long)fixed) / p.slot_bytes;
     if (slots > kMaxSlots) slots = kMaxSlots;
@@ -588,19 +703,12 @@ static coreinfer_status decode_stack_b1(const coreinfer_layer* layers, int L, co
     p.ybuf = (float*)((uint8_t*)workspace + kCtrlBytes);
 
     // Control words and the reduction targets start at zero.
-    if (L > 1) {
-        CI_CUDA(cudaMemsetAsync(workspace, 0, kCtrlBytes + (size_t)(L - 1) * d_model * sizeof(float), st));
-    } else {
-        CI_CUDA(cudaMemsetAsync(workspace, 0, kCtrlBytes, st));
-        CI_CUDA(cudaMemsetAsync(y_last, 0, (size_t)d_model * sizeof(float), st));
-        if (y_layers) CI_CUDA(cudaMemsetAsync(y_layers, 0, (size_t)d_model * sizeof(float), st));
-    }
-    const bool coop = L > 1;
+    CI_CUDA(cudaMemsetAsync(workspace, 0, b1_workspace_bytes(d_model), st));
     if (dtype == COREINFER_BF16)
-        return gated ? launch_vpt<__nv_bfloat16, true>(vpt, p, G, smem, coop, st)
-                     : launch_vpt<__nv_bfloat16, false>(vpt, p, G, smem, coop, st);
-    return gated ? launch_vpt<float, true>(vpt, p, G, smem, coop, st)
-                 : launch_vpt<float, false>(vpt, p, G, smem, coop, st);
+        return gated ? launch_shape<__nv_bfloat16, true>(groups, vpt, p, G, smem, st)
+                     : launch_shape<__nv_bfloat16, false>(groups, vpt, p, G, smem, st);
+    return gated ? launch_shape<float, true>(groups, vpt, p, G, smem, st)
+                 : launch_shape<float, false>(groups, vpt, p, G, smem, st);
 }
 
 // decode_batch.cu
@@ -617,7 +725,7 @@ extern "C" {
 size_t coreinfer_ffn_decode_workspace_bytes(int32_t batch, int32_t d_model, int32_t K)
 {
     if (batch < 1 || d_model < 1 || K < 1) return 0;
-    if (batch == 1) return kCtrlBytes;
+    if (batch == 1) return b1_workspace_bytes(d_model);
     return kCtrlBytes + (size_t)batch * (size_t)K * sizeof(float);   // h [batch, K]
 }
 
@@ -625,7 +733,7 @@ size_t coreinfer_ffn_decode_stack_workspace_bytes(int32_t L, int32_t batch, int3
 {
     (void)K_max;
     if (L < 1 || batch < 1 || d_model < 1) return 0;
-    return kCtrlBytes + (size_t)L * (size_t)batch * (size_t)d_model * sizeof(float);
+    return (size_t)batch * b1_workspace_bytes(d_model);
 }
 
 coreinfer_status coreinfer_ffn_decode(const void* x, int32_t batch, coreinfer_dtype dtype,
@@ -679,10 +787,10 @@ coreinfer_status coreinfer_ffn_decode_stack(const coreinfer_layer* layers, int32
 // handed every free byte of HBM to its own pools at start-up, a plug-in that runs inside a host
 // framework which forbids cudaMalloc on its threads because the call synchronises the whole
 // device, a latency-critical loop in which an allocator call is not acceptable.  For them the
-// scratch of the stack kernel (control words + the per-layer reduction targets) lives in a
+// scratch of the stack kernel (control words + the rotating reduction targets) lives in a
 // fixed array inside the library image.  The array costs kNoAllocScratchBytes of HBM on every
 // GPU that loads the library, for the life of the process.
-constexpr size_t kNoAllocScratchBytes = 4u << 20;   // 4 MiB: L * d_model * 4 + 256 must fit
+constexpr size_t kNoAllocScratchBytes = 256u << 10;   // 256 KiB: 256 + 24 * d_model bytes must fit
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
 
 // The array's name is only a handle on the host; its device address comes from
@@ -722,8 +830,8 @@ coreinfer_status coreinfer_ffn_decode_stack_noalloc(const coreinfer_layer* layer
     const size_t need = coreinfer_ffn_decode_stack_workspace_bytes(L, batch, d_model, 0);
     if (need > kNoAllocScratchBytes)
         CI_FAIL(COREINFER_ERR_UNSUPPORTED,
-                "L = %d, d_model = %d need %zu bytes of scratch; the built-in scratch holds %zu "
-                "(use coreinfer_ffn_decode_stack with a workspace)", L, d_model, need, kNoAllocScratchBytes);
+                "d_model = %d needs %zu bytes of scratch; the built-in scratch holds %zu "
+                "(use coreinfer_ffn_decode_stack with a workspace)", d_model, need, kNoAllocScratchBytes);
     void* scratch = nullptr;
     s = noalloc_scratch_ptr(&scratch);
     if (s != COREINFER_OK) return s;
