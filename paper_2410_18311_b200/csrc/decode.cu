@@ -47,6 +47,7 @@ struct LayerDev {
 
 struct DecodeParams {
     int L, d, nv, row_bytes, slot_bytes, n_slots, rmax;
+    int ysum_ofs;       // shared-memory offset of the two-group hand-over buffer
     const void* x0;
     float* y_last;
     float* y_layers;
@@ -208,7 +209,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
     constexpr int NMAT = GATED ? 2 : 1;
     constexpr int NC = NG * kGroupThreads;           // consumer threads
     constexpr int BATCH = batch_for(NG, VPT);        // ring items per batch
-    constexpr int FLUSH = 8 / BATCH;                 // own up batches per cross-lane reduction
+    constexpr int FLUSH = 16 / BATCH;                // own up batches per cross-lane reduction (16 row sums)
 
     extern __shared__ __align__(128) uint8_t smem[];
     uint8_t* ring = smem;
@@ -218,6 +219,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
     float* h_s = red + NMAT * kGroupWarps * p.rmax;                 // [rmax]
     float* ss_red = h_s + p.rmax;                                   // [NG][kGroupWarps]
     volatile int* abort_flag = reinterpret_cast<volatile int*>(ss_red + NG * kGroupWarps);
+    float* ysum = reinterpret_cast<float*>(smem + p.ysum_ofs);      // [NG == 2 ? VPT * 256 * EPV : 0]
 
     const int tid = threadIdx.x;
     const int G = gridDim.x;
@@ -324,11 +326,23 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
     // wait for the next n items, pull them into registers (q[j][i] = vector i of item j), free them
     auto fetch = [&](uint4 (&q)[BATCH][VPT], int n) {
         {
-            int sl = slot;
-            uint32_t ph = phase;
-            for (int j = 0; j < n; ++j) {
-                wait_slot(smem_u32(&full_bar[sl]), ph, abort_flag, p.ctrl);
-                if (++sl == NS) { sl = 0; ph ^= 1u; }
+            // test all barriers of the batch back to back (the tests overlap); only if one is
+            // not complete yet fall back to the bounded waits, one by one
+            bool ready = true;
+#pragma unroll
+            for (int j = 0; j < BATCH; ++j) {
+                int sl = slot + (j < n ? j : 0);
+                uint32_t ph = phase;
+                if (sl >= NS) { sl -= NS; ph ^= 1u; }
+                ready &= mbar_try_wait(smem_u32(&full_bar[sl]), ph);
+            }
+            if (!ready) {
+                int sl = slot;
+                uint32_t ph = phase;
+                for (int j = 0; j < n; ++j) {
+                    wait_slot(smem_u32(&full_bar[sl]), ph, abort_flag, p.ctrl);
+                    if (++sl == NS) { sl = 0; ph ^= 1u; }
+                }
             }
         }
         if (n == BATCH) {
@@ -372,9 +386,9 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
         // ------------------------------------------------ up (+ gate) phase --
         {
             const int nb = (n_up + BATCH - 1) / BATCH;
-            float part[8];
+            float part[16];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) part[j] = 0.f;
+            for (int j = 0; j < 16; ++j) part[j] = 0.f;
             int own = 0;                          // own batches accumulated in part[]
             int first_b = 0;                      // first of them
             for (int b = 0; b < nb; ++b) {
@@ -401,18 +415,26 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
                     }
                 }
                 ++own;
-                const bool flush = own == FLUSH || b + NG >= nb;
-                if (flush) {
-                    const float tot = warp_reduce8(part, lane);
+                if (own == FLUSH || b + NG >= nb) {
+                    // two independent 8-value reductions (their shuffles interleave)
+                    float lo[8], hi[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) { lo[j] = part[j]; hi[j] = part[8 + j]; }
+                    const float tot_lo = warp_reduce8(lo, lane);
+                    const float tot_hi = warp_reduce8(hi, lane);
                     if ((lane & 3) == 0) {
                         const int vi = ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);
-                        const int f = vi / BATCH, j = vi % BATCH;          // own batch f of the window, item j
-                        const int item = (first_b + f * NG) * BATCH + j;   // position in the up phase
-                        if (f < own && item < n_up)
-                            red[((item % NMAT) * kGroupWarps + gw) * p.rmax + item / NMAT] = tot;
+#pragma unroll
+                        for (int half = 0; half < 2; ++half) {
+                            const int pi = half * 8 + vi;                      // index in part[]
+                            const int f = pi / BATCH, j = pi % BATCH;          // own batch f of the window, item j
+                            const int item = (first_b + f * NG) * BATCH + j;   // position in the up phase
+                            if (f < own && item < n_up)
+                                red[((item % NMAT) * kGroupWarps + gw) * p.rmax + item / NMAT] = half ? tot_hi : tot_lo;
+                        }
                     }
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) part[j] = 0.f;
+                    for (int j = 0; j < 16; ++j) part[j] = 0.f;
                     own = 0;
                 }
             }
@@ -475,31 +497,43 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
         }
 
         // ----------------------------------------- cross-CTA sum of partial y --
-        // Every group adds its partial into one of kYCopies copies of the layer's target (adds to
+        // Every CTA adds its partial into one of kYCopies copies of the layer's target (adds to
         // one address are serialised in L2, so they are spread); after the grid barrier every
         // thread sums the copies for its columns.  Targets rotate over three buffers: while layer
         // l's is read, the one layer l+2 will use is cleared (last read before the barrier of l).
         const bool last = (l == p.L - 1);
         float* ybase = p.ybuf + (size_t)(l % kYBuffers) * kYCopies * d;
-        float* ytarget = ybase + (size_t)((cta + grp) & (kYCopies - 1)) * d;
+        float* ytarget = ybase + (size_t)(cta & (kYCopies - 1)) * d;
+        if (NG == 2) {            // one sum per CTA leaves the chip: group 1 hands its partial to group 0
+            if (grp == 1) {
 #pragma unroll
-        for (int i = 0; i < VPT; ++i) {
-            const int v = gt + i * kGroupThreads;
-            if (v < nv) {
+                for (int i = 0; i < VPT; ++i)
 #pragma unroll
-                for (int c = 0; c < PAIRS; c += 2)
-                    red_add_v4(ytarget + (size_t)v * EPV + 2 * c, yacc[i][c].x, yacc[i][c].y, yacc[i][c + 1].x,
-                               yacc[i][c + 1].y);
+                    for (int c = 0; c < PAIRS; c += 2)
+                        *reinterpret_cast<float4*>(ysum + (size_t)(gt + i * kGroupThreads) * EPV + 2 * c) =
+                            make_float4(yacc[i][c].x, yacc[i][c].y, yacc[i][c + 1].x, yacc[i][c + 1].y);
+            }
+            named_bar_sync(1, NC);
+        }
+        if (grp == 0) {
+#pragma unroll
+            for (int i = 0; i < VPT; ++i) {
+                const int v = gt + i * kGroupThreads;
+                if (v < nv) {
+#pragma unroll
+                    for (int c = 0; c < PAIRS; c += 2) {
+                        float4 t = make_float4(yacc[i][c].x, yacc[i][c].y, yacc[i][c + 1].x, yacc[i][c + 1].y);
+                        if (NG == 2) {
+                            const float4 o = *reinterpret_cast<const float4*>(ysum + (size_t)v * EPV + 2 * c);
+                            t.x += o.x; t.y += o.y; t.z += o.z; t.w += o.w;
+                        }
+                        red_add_v4(ytarget + (size_t)v * EPV + 2 * c, t.x, t.y, t.z, t.w);
+                    }
+                }
             }
         }
 
         grid_barrier(p.ctrl, (unsigned)(l + 1) * (unsigned)G, abort_flag, NC);
-
-        {
-            float4* z = reinterpret_cast<float4*>(p.ybuf + (size_t)((l + 2) % kYBuffers) * kYCopies * d);
-            const int n4 = kYCopies * d / 4;
-            for (int i = cta * NC + tid; i < n4; i += G * NC) z[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-        }
 
         // ------------------------- next input: (x + y) / rms(x + y), rounded --
         float ss = 0.f;
@@ -532,6 +566,11 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
                 }
             }
         }
+        {   // clear the target that layer l + 2 will use
+            float4* z = reinterpret_cast<float4*>(p.ybuf + (size_t)((l + 2) % kYBuffers) * kYCopies * d);
+            const int n4 = kYCopies * d / 4;
+            for (int i = cta * NC + tid; i < n4; i += G * NC) z[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
         if (last) break;
         // every group holds all columns, so each forms the norm on its own (same sums, same order)
 #pragma unroll
@@ -558,6 +597,12 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
 }
 
 // ------------------------------------------------------------------- host ---
+// fp32 hand-over buffer of the two-group kernels: every thread of a group stores all its columns
+static size_t ysum_smem_bytes(int groups, int vpt, size_t esize)
+{
+    return groups == 2 ? (size_t)vpt * kGroupThreads * (16 / esize) * sizeof(float) : 0;
+}
+
 static size_t fixed_smem_bytes(int rmax, bool gated, int groups)
 {
     size_t b = 2 * kMaxSlots * sizeof(uint64_t);
@@ -688,13 +733,15 @@ static coreinfer_status decode_stack_b1(const coreinfer_layer* layers, int L, co
                 d_model, 8 * kGroupThreads * 16);
     const int vpt = groups == 2 ? ((p.nv + kGroupThreads - 1) / kGroupThreads <= 1 ? 1 : 2) : vpt_for(p.nv);
     const int batch = batch_for(groups, groups == 2 ? vpt : (vpt <= 3 ? 3 : vpt));
-    const size_t fixed = fixed_smem_bytes(p.rmax, gated, groups);
+    const size_t fixed0 = fixed_smem_bytes(p.rmax, gated, groups);
+    const size_t fixed = fixed0 + ysum_smem_bytes(groups, vpt, esize);
     if (fixed + (size_t)batch * p.slot_bytes > (size_t)di.smem_optin)
         CI_FAIL(COREINFER_ERR_UNSUPPORTED, "K = %d, d_model = %d do not fit in shared memory", Kmax, d_model);
     long long slots = ((long long)di.smem_optin - (long long)fixed) / p.slot_bytes;
     if (slots > kMaxSlots) slots = kMaxSlots;
     p.n_slots = (int)slots;
     const size_t smem = fixed + (size_t)p.n_slots * p.slot_bytes;
+    p.ysum_ofs = (int)((size_t)p.n_slots * p.slot_bytes + fixed0);
     p.x0 = x0;
     p.y_last = y_last;
     p.y_layers = y_layers;
