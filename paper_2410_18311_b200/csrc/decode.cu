@@ -739,6 +739,9 @@ static coreinfer_status decode_stack_b1(const coreinfer_layer* layers, int L, co
         CI_FAIL(COREINFER_ERR_UNSUPPORTED, "K = %d, d_model = %d do not fit in shared memory", Kmax, d_model);
     long long slots = ((long long)di.smem_optin - (long long)fixed) / p.slot_bytes;
     if (slots > kMaxSlots) slots = kMaxSlots;
+    // With two groups a slot must always come back to the same group (a group never waits on the
+    // other's items, so only then can it never be a full ring pass ahead of a barrier it tests).
+    if (groups == 2 && slots >= 2 * batch) slots -= slots % (2 * batch);
     p.n_slots = (int)slots;
     const size_t smem = fixed + (size_t)p.n_slots * p.slot_bytes;
     p.ysum_ofs = (int)((size_t)p.n_slots * p.slot_bytes + fixed0);
