@@ -128,7 +128,7 @@ __device__ __forceinline__ bool wait_slot(uint32_t bar, uint32_t parity, volatil
     if (*abort_flag) return false;
     const long long t0 = clock64();
     for (;;) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (mbar_try_wait_parked(bar, parity, 4000u)) return true;
         if (*abort_flag) return false;
         if (clock64() - t0 > kWaitCycles) {
             *abort_flag = 1;
@@ -151,6 +151,7 @@ __device__ __forceinline__ void grid_barrier(unsigned* ctrl, unsigned target, vo
         unsigned it = 0;
         for (;;) {
             if (ld_acquire_gpu(&ctrl[1]) >= target) break;
+            __nanosleep(32);
             if ((++it & 255u) == 0u) {             // now and then: has another CTA given up? out of time?
                 if (ld_acquire_gpu(&ctrl[0]) != kStatusOk) { *abort_flag = 1; break; }
                 if (clock64() - t0 > kWaitCycles) {
