@@ -27,8 +27,10 @@ METRIC = "core-sparse decode tokens/s at batch 1; achieved HBM GB/s vs B200 peak
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode_stack_kernel launch at the bench
-# workload, from the ncu capture summarised in profiles/ (None until captured for this kernel)
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+# workload: measured by ncu on a 4-layer launch of the same shapes (219.0 MB) and scaled by the
+# layer count, since every layer streams its own weights (profiles/decode_stack_kernel_opt6.7b.md).
+# Set to None whenever the kernel changes until the capture is repeated.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"opt6.7b": 219.0e6 / 4 * 32}
 
 
 def parse_args():
@@ -385,7 +387,7 @@ def run_ours(args, cfg):
         "roofline": {"bound": "hbm", "kernel": "decode_stack_kernel", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_source": "of " + peak_src,
                      "bytes_per_launch": bytes_tok, "launch_us": launch_s * 1e6,
-                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH},
+                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(cfg.name)},
         "e2e": e2e,
         "gpu_launches": args.steps * (cfg.L * (stack.SELECT_KERNELS_PER_LAYER + stack.COMPACT_KERNELS_PER_LAYER)
                                       + steps_tok * stack.DECODE_KERNELS_PER_TOKEN),
@@ -393,7 +395,7 @@ def run_ours(args, cfg):
         "context": "paper (TITAN Xp, end to end, other workload): 10.33x over HuggingFace, 2.72x over PowerInfer",
     }
     if not args.no_cpu_baseline and world == 1:
-        line["cpu_baseline"] = oracle_sample(cfg, n_layers=2, n_tokens=4)
+        line["cpu_baseline"] = oracle_sample(cfg, n_layers=4, n_tokens=min(cfg.decode_steps, 256))
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
