@@ -12,8 +12,8 @@
 //                        membership counters of Eq. 3 live in its registers: no atomics.
 //                        At the end each CTA writes its counters as one u16 row.
 //   select_count_kernel  f[n] = sum over CTAs of those rows (int32).
-//   select_top_kernel    one CTA: the K-th largest count c* by bisection on the count value,
-//                        then an index-ordered scan admits f > c*, and the lowest-index
+//   select_top_kernel    one CTA: the K-th largest count c* by a histogram search on the count
+//                        value, then an index-ordered scan admits f > c*, and the lowest-index
 //                        f == c* until K are taken, and writes them in ascending index.
 #include "common.cuh"
 
@@ -285,54 +285,77 @@ select_rows_kernel(const float* __restrict__ act, int T, int N, long long ld, do
     }
 }
 
-__global__ void __launch_bounds__(256)
+// f[n] = sum over the CTAs' u16 rows.  A block covers 32 groups of 4 neurons; its 8 warps take
+// every 8th row each (so the loads of a column group are spread over 8 threads) and meet in
+// shared memory.
+constexpr int kCountCols = 32;
+constexpr int kCountSlices = 8;
+
+__global__ void __launch_bounds__(kCountCols * kCountSlices)
 select_count_kernel(const uint16_t* __restrict__ partial, int G, int n4, int N, int32_t* __restrict__ f)
 {
-    const int v = blockIdx.x * blockDim.x + threadIdx.x;   // one group of 4 neurons per thread
-    if (v * 4 >= N) return;
-    int c0 = 0, c1 = 0, c2 = 0, c3 = 0;
-    for (int g = 0; g < G; ++g) {
-        const uint2 w = reinterpret_cast<const uint2*>(partial + (size_t)g * n4)[v];
-        c0 += w.x & 0xffff; c1 += w.x >> 16; c2 += w.y & 0xffff; c3 += w.y >> 16;
+    __shared__ int4 acc[kCountSlices][kCountCols];
+    const int col = threadIdx.x & (kCountCols - 1);
+    const int slice = threadIdx.x / kCountCols;
+    const int v = blockIdx.x * kCountCols + col;           // group of 4 neurons
+    int4 c = make_int4(0, 0, 0, 0);
+    if (v * 4 < n4) {
+        for (int g = slice; g < G; g += kCountSlices) {
+            const uint2 w = reinterpret_cast<const uint2*>(partial + (size_t)g * n4)[v];
+            c.x += w.x & 0xffff; c.y += w.x >> 16; c.z += w.y & 0xffff; c.w += w.y >> 16;
+        }
     }
-    const int n = v * 4;
-    f[n] = c0;
-    if (n + 1 < N) f[n + 1] = c1;
-    if (n + 2 < N) f[n + 2] = c2;
-    if (n + 3 < N) f[n + 3] = c3;
+    acc[slice][col] = c;
+    __syncthreads();
+    if (slice == 0 && v * 4 < N) {
+#pragma unroll
+        for (int sl = 1; sl < kCountSlices; ++sl) {
+            const int4 o = acc[sl][col];
+            c.x += o.x; c.y += o.y; c.z += o.z; c.w += o.w;
+        }
+        const int n = v * 4;
+        f[n] = c.x;
+        if (n + 1 < N) f[n + 1] = c.y;
+        if (n + 2 < N) f[n + 2] = c.z;
+        if (n + 3 < N) f[n + 3] = c.w;
+    }
 }
 
-// One CTA.  Thread t owns the contiguous neurons [t*C, (t+1)*C).
+// One CTA.  Thread t owns the contiguous neurons [t*C, (t+1)*C).  The K-th largest count c* is
+// found with the same histogram search as a row threshold (12 high bits of the count, then, for
+// counts of 4096 and more, the low bits); the members are then f > c* plus the lowest-index
+// f == c* until K are taken, written in ascending index with two block scans.
 __global__ void __launch_bounds__(kSelThreads, 1)
 select_top_kernel(const int32_t* __restrict__ f, int N, int K, int T, int32_t* __restrict__ S)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     int* fs = reinterpret_cast<int*>(smem);                               // [N]
-    SelShared* sh = reinterpret_cast<SelShared*>(fs + ((N + 3) & ~3));
+    int* hist = fs + ((N + 3) & ~3);                                      // [kSelBins]
+    SelShared* sh = reinterpret_cast<SelShared*>(hist + kSelBins);
     const int tid = threadIdx.x;
     for (int i = tid; i < N; i += kSelThreads) fs[i] = f[i];
-    __syncthreads();
     const int C = (N + kSelThreads - 1) / kSelThreads;
     const int n0 = min(tid * C, N), n1 = min(n0 + C, N);
 
-    // c* = smallest c with #(f > c) < K  (the K-th largest count), by bisection on [0, T]
-    int lo = 0, hi = T;                 // invariant: #(f > hi) < K (counts never exceed T)
-    int above_hi = 0;
-    while (lo < hi) {
-        const int mid = (lo + hi) >> 1;
-        int c = 0;
-        for (int n = n0; n < n1; ++n) c += fs[n] > mid ? 1 : 0;
-        int tot;
-        block_excl_scan(c, sh, &tot);
-        if (tot < K) { hi = mid; above_hi = tot; } else { lo = mid + 1; }
+    int shift = 0;                      // counts lie in [0, T]; the first pass looks at f >> shift
+    while ((T >> shift) >= kSelBins) ++shift;
+    int cstar = 0, above = 0, need = K;
+    for (int pass = 0; pass < (shift > 0 ? 2 : 1); ++pass) {
+        for (int i = tid; i < kSelBins; i += kSelThreads) hist[i] = 0;
+        __syncthreads();
+        for (int n = n0; n < n1; ++n) {
+            const int v = fs[n];
+            if (pass == 0) atomicAdd(&hist[v >> shift], 1);
+            else if ((v >> shift) == (cstar >> shift)) atomicAdd(&hist[v & ((1 << shift) - 1)], 1);
+        }
+        __syncthreads();
+        find_bin(hist, need, false, 0.0, sh);
+        cstar |= pass == 0 ? (sh->bin << shift) : sh->bin;
+        above += sh->above;
+        need -= sh->above;
+        __syncthreads();
     }
-    const int cstar = lo;
-    {   // #(f > c*) (above_hi is stale if the loop never lowered hi to c*)
-        int c = 0;
-        for (int n = n0; n < n1; ++n) c += fs[n] > cstar ? 1 : 0;
-        block_excl_scan(c, sh, &above_hi);
-    }
-    const int need = K - above_hi;      // how many f == c* are admitted, lowest index first
+    // need = how many f == c* are admitted, lowest index first
 
     int ce = 0;
     for (int n = n0; n < n1; ++n) ce += fs[n] == cstar ? 1 : 0;
@@ -440,10 +463,10 @@ coreinfer_status coreinfer_select_core(const void* act, coreinfer_dtype act_dtyp
 #undef CI_ROWS
     if (s != COREINFER_OK) return s;
 
-    select_count_kernel<<<(n4 / 4 + 255) / 256, 256, 0, st>>>(partial, G, n4, d_ff, f);
+    select_count_kernel<<<(n4 / 4 + kCountCols - 1) / kCountCols, kCountCols * kCountSlices, 0, st>>>(partial, G, n4, d_ff, f);
     CI_CUDA(cudaGetLastError());
 
-    const size_t smem_top = (size_t)n4 * sizeof(int) + sizeof(SelShared) + 16;
+    const size_t smem_top = (size_t)n4 * sizeof(int) + kSelBins * sizeof(int) + sizeof(SelShared) + 16;
     CI_CUDA(cudaFuncSetAttribute(select_top_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_top));
     select_top_kernel<<<1, kSelThreads, smem_top, st>>>(f, d_ff, K, T, core_idx);
     CI_CUDA(cudaGetLastError());
