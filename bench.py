@@ -43,6 +43,10 @@ def parse_args():
     ap.add_argument("--no-dense", action="store_true", help="skip the dense (alpha = beta = 1) comparison")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--decode-only", type=int, default=0, metavar="LAYERS",
+                    help="profiling target: only decode launches through the first LAYERS layers of the config "
+                         "on random compacted weights (small enough for an ncu capture); prints a short JSON line")
+    ap.add_argument("--tokens", type=int, default=2, help="decode launches per step in --decode-only mode")
     return ap.parse_args()
 
 
@@ -401,10 +405,48 @@ def run_ours(args, cfg):
         dist.destroy_process_group()
 
 
+def run_decode_only(args, cfg):
+    """A few launches of the decode kernel alone, on a stack cut to --decode-only layers: the target
+    of the full-counter ncu capture (a whole 32-layer launch is too long to replay 40 times)."""
+    import torch
+    import paper_2410_18311_b200 as ci
+    from paper_2410_18311_b200 import _build, workloads as wl
+    _build.build()
+    cfg = cfg.with_(L=args.decode_only)
+    K = ci.coreinfer_count(cfg.beta, cfg.d_ff)
+    layers = [wl.compacted_weights_random(cfg, l, K, device="cuda") for l in range(cfg.L)]
+    arr = ci.binding.make_layers([(u, g, dn, None, None) for (u, g, dn) in layers])
+    kind = ci.FFN_RELU_GATED if cfg.gated else ci.FFN_RELU
+    xs = torch.cat([wl.decode_input(cfg, s, device="cuda") for s in range(args.tokens)], dim=0)
+    ys = torch.empty((args.tokens, cfg.d_model), device="cuda")
+    ws = torch.empty(ci.coreinfer_ffn_decode_stack_workspace_bytes(cfg.L, 1, cfg.d_model, K), dtype=torch.uint8,
+                     device="cuda")
+
+    def step():
+        for t in range(args.tokens):
+            ci.coreinfer_ffn_decode_stack(arr, xs[t:t + 1], kind, ys[t:t + 1], None, None, ws)
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    ci.coreinfer_workspace_status(ws)
+    us = e0.elapsed_time(e1) * 1e3 / (args.steps * args.tokens)
+    nbytes = cfg.L * cfg.n_mat * K * cfg.d_model * cfg.esize
+    print(json.dumps({"mode": "decode-only", "workload": cfg.name, "layers": cfg.L, "K": K, "us_per_launch": us,
+                      "bytes_per_launch": nbytes, "gbs": nbytes / us / 1e3}), flush=True)
+
+
 def main():
     args = parse_args()
     from paper_2410_18311_b200 import workloads as wl
     cfg = wl.CONFIGS[args.config]
+    if args.decode_only > 0:
+        return run_decode_only(args, cfg)
     if args.impl == "reference":
         run_reference(args, cfg)
     else:
