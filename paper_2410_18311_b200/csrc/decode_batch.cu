@@ -1,5 +1,6 @@
 // Decode FFN over compacted weights for 2..8 sequences that share one core set
-// (Section 4.2 applied to a small batch).  Two plain streaming kernels:
+// (Section 4.2 applied to a small batch): the plain kernels, used for fp32 and for bf16 rows the
+// tensor-core kernel (decode_batch_mma.cu) is not built for.  Two streaming kernels:
 //   up:   one warp per core neuron forms h[b, k] for every sequence b (fp32, kept in
 //         the caller's workspace, [batch, K]);
 //   down: CTAs tile (column block, neuron range), accumulate partial y[b, :] in
@@ -174,6 +175,10 @@ static coreinfer_status run_t(int batch, const void* x, bool gated, int d_model,
     }
 }
 
+// decode_batch_mma.cu: tensor-core kernel for bf16 rows of up to 4096 columns
+coreinfer_status decode_batched_mma(const void* x, int batch, bool gated, int d_model, const coreinfer_layer& ly,
+                                    float* y, unsigned* status, const DeviceInfo& di, cudaStream_t st);
+
 coreinfer_status decode_batched(const void* x, int batch, coreinfer_dtype dtype, coreinfer_ffn_kind kind,
                                 int d_model, const coreinfer_layer& ly, float* y, void* workspace,
                                 cudaStream_t st)
@@ -182,7 +187,11 @@ coreinfer_status decode_batched(const void* x, int batch, coreinfer_dtype dtype,
     coreinfer_status s = device_info(&di);
     if (s != COREINFER_OK) return s;
     const bool gated = kind == COREINFER_FFN_RELU_GATED;
-    CI_CUDA(cudaMemsetAsync(workspace, 0, kCtrlBytesB, st));   // status word: nothing here can time out
+    CI_CUDA(cudaMemsetAsync(workspace, 0, kCtrlBytesB, st));   // status word
+    if (dtype == COREINFER_BF16) {
+        s = decode_batched_mma(x, batch, gated, d_model, ly, y, (unsigned*)workspace, di, st);
+        if (s != COREINFER_ERR_UNSUPPORTED) return s;          // otherwise: shape not built there, use the plain kernels
+    }
     float* h = (float*)((uint8_t*)workspace + kCtrlBytesB);
     if (dtype == COREINFER_BF16) return run_t<__nv_bfloat16>(batch, x, gated, d_model, ly, y, h, st);
     return run_t<float>(batch, x, gated, d_model, ly, y, h, st);

@@ -1,0 +1,374 @@
+// Decode FFN over compacted weights for 2..8 sequences that share one core set (Section 4.2
+// applied to a small batch), bf16, one layer per launch.
+//
+// With eight sequences the work per weight byte is eight times that of batch 1 and the fp32
+// pipes would become the limit, so here the sequences sit on the N = 8 side of
+// mma.sync.m16n8k16 (bf16 inputs, fp32 accumulate): this is the one place where the path is a
+// real dense contraction.  The streaming structure is that of the batch-1 kernel: one CTA per
+// SM owns a slab of neurons, a producer warp fills a ring of shared-memory slots with 1-D bulk
+// copies (slot stride = row + 16 bytes, so that the 8 rows of an ldmatrix tile fall into
+// different banks), and sixteen consumer warps each own d_model / 16 columns.
+//   up:   A = 16 weight rows (8 up + 8 gate rows when gated) x 16 columns from the ring,
+//         B = x^T fragments kept in registers; the sixteen warps' 16 x 8 partial tiles are
+//         added in shared memory, then bias + ReLU (or gate product) gives h in fp32.
+//   down: A = the transposed view (ldmatrix.trans) of 16 down rows, B = h split exactly into
+//         three bf16 parts (hi + mid + lo = the fp32 value), three MMAs per tile; the
+//         [d_model / 16 columns] x [8 sequences] accumulators stay in registers for the slab.
+//   out:  tiles are turned in shared memory and added to y with vector reductions.
+// Every wait is bounded as in the batch-1 kernel.
+#include "common.cuh"
+
+namespace coreinfer {
+
+constexpr int kMmaWarps = 16;
+constexpr int kMmaThreads = kMmaWarps * 32;
+constexpr int kMmaBlock = kMmaThreads + 32;
+constexpr int kMmaMaxSlots = 64;
+constexpr int kMmaMaxTiles = 16;                    // d_model / 16 warps / 16 columns <= 16  ->  d_model <= 4096
+constexpr long long kMmaWaitCycles = 3000000000LL;
+
+struct MmaParams {
+    const uint8_t* up;
+    const uint8_t* gate;
+    const uint8_t* down;
+    const __nv_bfloat16* bup;
+    const __nv_bfloat16* bdown;
+    const __nv_bfloat16* x;     // [B][d]
+    float* y;                   // [B][d], zero on entry
+    unsigned* status;
+    int K, d, B, row_bytes, slot_stride, n_slots, rpad;
+};
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&a)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3]) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&a)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3]) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ bool mma_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned* status)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    const long long t0 = clock64();
+    for (;;) {
+        if (mbar_try_wait_parked(bar, parity, 4000u)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kMmaWaitCycles) {
+            *abort_flag = 1;
+            atomicMax(status, (unsigned)kStatusTimeout);
+            return false;
+        }
+    }
+}
+
+template <bool GATED>
+__global__ void __launch_bounds__(kMmaBlock, 1)
+decode_batch_mma_kernel(const MmaParams p)
+{
+    constexpr int NMAT = GATED ? 2 : 1;
+    constexpr int RU = 16 / NMAT;                    // neurons per up unit (16 tile rows)
+
+    extern __shared__ __align__(128) uint8_t smem[];
+    const int NS = p.n_slots;
+    uint8_t* ring = smem;
+    uint8_t* zero_row = ring + (size_t)NS * p.slot_stride;                       // a row of zeros for padded tile rows
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(zero_row + p.slot_stride);
+    uint64_t* empty_bar = full_bar + kMmaMaxSlots;
+    float* scratch = reinterpret_cast<float*>(empty_bar + kMmaMaxSlots);         // [16 warps][128]: partial tiles / output staging
+    __nv_bfloat16* hpart = reinterpret_cast<__nv_bfloat16*>(scratch + kMmaWarps * 128);   // [3][8][rpad]
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(hpart + 3 * 8 * p.rpad);
+
+    const int tid = threadIdx.x;
+    const int G = gridDim.x, cta = blockIdx.x;
+    const int k0 = (int)(((long long)cta * p.K) / G), k1 = (int)(((long long)(cta + 1) * p.K) / G);
+    const int n = k1 - k0;
+    const int n_up_units = (n + RU - 1) / RU;
+    const int n_dn_units = (n + 15) / 16;
+
+    if (tid == 0) {
+        for (int s = 0; s < NS; ++s) {
+            mbar_init(smem_u32(&full_bar[s]), 1);
+            mbar_init(smem_u32(&empty_bar[s]), kMmaWarps);
+        }
+        *abort_flag = 0;
+        mbar_fence_init();
+    }
+    for (int i = tid; i < p.slot_stride / 16; i += kMmaBlock) reinterpret_cast<uint4*>(zero_row)[i] = make_uint4(0, 0, 0, 0);
+    for (int i = tid; i < 3 * 8 * p.rpad; i += kMmaBlock) hpart[i] = __float2bfloat16(0.f);
+    __syncthreads();
+
+    // ======================================================== producer warp ==
+    if (tid >= kMmaThreads) {
+        const int lane = tid - kMmaThreads;
+        const int round_max = NS < 8 ? NS : 8;
+        const int n_up_items = n * NMAT;
+        const int total = n_up_items + n;
+        int slot0 = 0;
+        uint32_t phase0 = 0;
+        long long issued = 0;
+        for (int q0 = 0; q0 < total; q0 += round_max) {
+            if (*abort_flag) break;
+            const int cnt = min(round_max, total - q0);
+            if (lane < cnt) {
+                const int q = q0 + lane;
+                const uint8_t* src;
+                if (q < n_up_items) {
+                    // unit u holds cnt_u up rows followed (gated) by the same neurons' gate rows
+                    const int u = q / (RU * NMAT);
+                    const int w = q - u * RU * NMAT;
+                    const int cnt_u = min(RU, n - u * RU);
+                    const int r = w % cnt_u, m = w / cnt_u;
+                    src = (m ? p.gate : p.up) + (size_t)(k0 + u * RU + r) * p.row_bytes;
+                } else {
+                    src = p.down + (size_t)(k0 + q - n_up_items) * p.row_bytes;
+                }
+                int sl = slot0 + lane;
+                uint32_t ph = phase0;
+                if (sl >= NS) { sl -= NS; ph ^= 1u; }
+                if (mma_wait(smem_u32(&empty_bar[sl]), ph ^ 1u, abort_flag, p.status)) {
+                    const uint32_t fb = smem_u32(&full_bar[sl]);
+                    mbar_arrive_expect_tx(fb, (uint32_t)p.row_bytes);
+                    bulk_g2s(smem_u32(ring + (size_t)sl * p.slot_stride), src, (uint32_t)p.row_bytes, fb);
+                }
+            }
+            __syncwarp();
+            slot0 += cnt;
+            if (slot0 >= NS) { slot0 -= NS; phase0 ^= 1u; }
+            issued += cnt;
+        }
+        for (int sl = lane; sl < NS; sl += 32) {      // leave only when nothing is in flight into this CTA
+            const long long uses = issued / NS + (sl < (int)(issued % NS) ? 1 : 0);
+            if (uses == 0) continue;
+            const uint32_t fb = smem_u32(&full_bar[sl]);
+            const uint32_t ph = (uint32_t)((uses - 1) & 1);
+            const long long t0 = clock64();
+            while (!mbar_try_wait(fb, ph))
+                if (clock64() - t0 > kMmaWaitCycles) { atomicMax(p.status, (unsigned)kStatusTimeout); break; }
+        }
+        return;
+    }
+
+    // ============================================================ consumers ==
+    const int lane = tid & 31, warp = tid >> 5;
+    const int JW = p.d / kMmaWarps;                   // columns of this warp (a multiple of 16)
+    const int jw = warp * JW;
+    const int ntile = JW / 16;                        // <= kMmaMaxTiles
+
+    // x^T fragments: B[k][n] = x[n][jw + 16 t + k]; lane holds k = 2 (lane % 4) + {0, 1} (+ 8), n = lane / 4
+    uint32_t xb[kMmaMaxTiles][2];
+    {
+        const int nb = lane >> 2;
+        const uint32_t* xrow = reinterpret_cast<const uint32_t*>(p.x + (size_t)(nb < p.B ? nb : 0) * p.d);
+#pragma unroll
+        for (int t = 0; t < kMmaMaxTiles; ++t) {
+            xb[t][0] = xb[t][1] = 0u;
+            if (t < ntile && nb < p.B) {
+                const int j = jw + t * 16 + (lane & 3) * 2;
+                xb[t][0] = xrow[j >> 1];
+                xb[t][1] = xrow[(j + 8) >> 1];
+            }
+        }
+    }
+
+    int slot = 0;
+    uint32_t phase = 0;
+    auto wait_items = [&](int cnt) {
+        int sl = slot;
+        uint32_t ph = phase;
+        for (int j = 0; j < cnt; ++j) {
+            mma_wait(smem_u32(&full_bar[sl]), ph, abort_flag, p.status);
+            if (++sl == NS) { sl = 0; ph ^= 1u; }
+        }
+    };
+    auto item_addr = [&](int j) -> uint32_t {
+        int sl = slot + j;
+        if (sl >= NS) sl -= NS;
+        return smem_u32(ring + (size_t)sl * p.slot_stride);
+    };
+    auto release_items = [&](int cnt) {       // cnt <= 16
+        __syncwarp();
+        if (lane < cnt && !*abort_flag) {
+            int sl = slot + lane;
+            if (sl >= NS) sl -= NS;
+            mbar_arrive(smem_u32(&empty_bar[sl]));
+        }
+        slot += cnt;
+        if (slot >= NS) { slot -= NS; phase ^= 1u; }
+    };
+    const uint32_t zero_addr = smem_u32(zero_row);
+
+    // ------------------------------------------------------ up (+ gate) units --
+    for (int u = 0; u < n_up_units; ++u) {
+        const int cnt = min(RU, n - u * RU);
+        wait_items(cnt * NMAT);
+        // tile row of this lane (for ldmatrix lane l addresses row l % 16, column half l / 16)
+        const int tr = lane & 15;
+        uint32_t rowaddr;
+        if (GATED) {
+            const int r = tr & 7, m = tr >> 3;
+            rowaddr = r < cnt ? item_addr(m * cnt + r) : zero_addr;
+        } else {
+            rowaddr = tr < cnt ? item_addr(tr) : zero_addr;
+        }
+        rowaddr += (uint32_t)(jw + 8 * (lane >> 4)) * 2u;
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int t = 0; t < kMmaMaxTiles; ++t) {
+            if (t < ntile) {
+                uint32_t a[4];
+                ldmatrix_x4(a, rowaddr + (uint32_t)t * 32u);
+                mma_bf16_16816(acc, a, xb[t][0], xb[t][1]);
+            }
+        }
+        release_items(cnt * NMAT);
+        // partial tile of this warp: rows m = lane / 4 (+ 8), sequences 2 (lane % 4) + {0, 1}
+        float* mine = scratch + warp * 128;
+        mine[(lane >> 2) * 8 + (lane & 3) * 2] = acc[0];
+        mine[(lane >> 2) * 8 + (lane & 3) * 2 + 1] = acc[1];
+        mine[((lane >> 2) + 8) * 8 + (lane & 3) * 2] = acc[2];
+        mine[((lane >> 2) + 8) * 8 + (lane & 3) * 2 + 1] = acc[3];
+        named_bar_sync(1, kMmaThreads);
+        if (tid < RU * 8) {
+            const int r = tid >> 3, nb = tid & 7;
+            float uu = 0.f, gg = 0.f;
+#pragma unroll
+            for (int w = 0; w < kMmaWarps; ++w) {
+                uu += scratch[w * 128 + r * 8 + nb];
+                if (GATED) gg += scratch[w * 128 + (r + 8) * 8 + nb];
+            }
+            float h = 0.f;
+            if (r < cnt) {
+                if (GATED) {
+                    h = fmaxf(gg, 0.f) * uu;
+                } else {
+                    if (p.bup) uu += __bfloat162float(p.bup[k0 + u * RU + r]);
+                    h = fmaxf(uu, 0.f);
+                }
+            }
+            // h = h1 + h2 + h3 exactly (three bf16 parts cover the 24-bit significand)
+            const __nv_bfloat16 h1 = __float2bfloat16_rn(h);
+            const float r1 = h - __bfloat162float(h1);
+            const __nv_bfloat16 h2 = __float2bfloat16_rn(r1);
+            const __nv_bfloat16 h3 = __float2bfloat16_rn(r1 - __bfloat162float(h2));
+            const int kk = u * RU + r;
+            hpart[(0 * 8 + nb) * p.rpad + kk] = h1;
+            hpart[(1 * 8 + nb) * p.rpad + kk] = h2;
+            hpart[(2 * 8 + nb) * p.rpad + kk] = h3;
+        }
+        named_bar_sync(1, kMmaThreads);
+    }
+
+    // --------------------------------------------------------------- down units --
+    float dacc[kMmaMaxTiles][4];
+#pragma unroll
+    for (int t = 0; t < kMmaMaxTiles; ++t) { dacc[t][0] = dacc[t][1] = dacc[t][2] = dacc[t][3] = 0.f; }
+    for (int ku = 0; ku < n_dn_units; ++ku) {
+        const int kk0 = ku * 16;
+        const int cnt = min(16, n - kk0);
+        wait_items(cnt);
+        // transposed tile: lane l addresses stored row k = 8 (l / 16) + l % 8, column block (l / 8) % 2
+        const int kr = ((lane >> 4) << 3) + (lane & 7);
+        uint32_t rowaddr = (kr < cnt ? item_addr(kr) : zero_addr) + (uint32_t)(jw + 8 * ((lane >> 3) & 1)) * 2u;
+        uint32_t hb[3][2];
+#pragma unroll
+        for (int s3 = 0; s3 < 3; ++s3) {
+            const uint32_t* hrow = reinterpret_cast<const uint32_t*>(hpart + (size_t)(s3 * 8 + (lane >> 2)) * p.rpad + kk0);
+            hb[s3][0] = hrow[lane & 3];
+            hb[s3][1] = hrow[(lane & 3) + 4];
+        }
+#pragma unroll
+        for (int t = 0; t < kMmaMaxTiles; ++t) {
+            if (t < ntile) {
+                uint32_t a[4];
+                ldmatrix_x4_trans(a, rowaddr + (uint32_t)t * 32u);
+                mma_bf16_16816(dacc[t], a, hb[0][0], hb[0][1]);
+                mma_bf16_16816(dacc[t], a, hb[1][0], hb[1][1]);
+                mma_bf16_16816(dacc[t], a, hb[2][0], hb[2][1]);
+            }
+        }
+        release_items(cnt);
+    }
+
+    // ---------------------------------------------------------------- output --
+    // dacc[t]: columns j = jw + 16 t + lane / 4 (+ 8), sequences 2 (lane % 4) + {0, 1}.  Turn each tile
+    // in this warp's scratch so that a lane owns 4 consecutive columns of one sequence.
+    float* st = scratch + warp * 128;            // [8 sequences][16 columns]
+    named_bar_sync(1, kMmaThreads);              // the up phase's last use of the scratch is over
+#pragma unroll
+    for (int t = 0; t < kMmaMaxTiles; ++t) {
+        if (t < ntile) {
+            const int jl = lane >> 2, nb = (lane & 3) * 2;
+            st[nb * 16 + jl] = dacc[t][0];
+            st[(nb + 1) * 16 + jl] = dacc[t][1];
+            st[nb * 16 + jl + 8] = dacc[t][2];
+            st[(nb + 1) * 16 + jl + 8] = dacc[t][3];
+            __syncwarp();
+            const int nn = lane >> 2, jq = (lane & 3) * 4;
+            float4 v = *reinterpret_cast<const float4*>(st + nn * 16 + jq);
+            const int j = jw + t * 16 + jq;
+            if (nn < p.B) {
+                if (cta == 0 && p.bdown) {
+                    v.x += __bfloat162float(p.bdown[j]);     v.y += __bfloat162float(p.bdown[j + 1]);
+                    v.z += __bfloat162float(p.bdown[j + 2]); v.w += __bfloat162float(p.bdown[j + 3]);
+                }
+                red_add_v4(p.y + (size_t)nn * p.d + j, v.x, v.y, v.z, v.w);
+            }
+            __syncwarp();
+        }
+    }
+}
+
+// Returns COREINFER_ERR_UNSUPPORTED (without setting an error text) when the shape is not built here.
+coreinfer_status decode_batched_mma(const void* x, int batch, bool gated, int d_model, const coreinfer_layer& ly,
+                                    float* y, unsigned* status, const DeviceInfo& di, cudaStream_t st)
+{
+    if (d_model % (kMmaWarps * 16) != 0 || d_model / (kMmaWarps * 16) > kMmaMaxTiles) return COREINFER_ERR_UNSUPPORTED;
+    MmaParams p;
+    p.up = (const uint8_t*)ly.w_up_c;
+    p.gate = (const uint8_t*)ly.w_gate_c;
+    p.down = (const uint8_t*)ly.w_downT_c;
+    p.bup = (const __nv_bfloat16*)ly.b_up_c;
+    p.bdown = (const __nv_bfloat16*)ly.b_down;
+    p.x = (const __nv_bfloat16*)x;
+    p.y = y;
+    p.status = status;
+    p.K = ly.K;
+    p.d = d_model;
+    p.B = batch;
+    p.row_bytes = d_model * 2;
+    p.slot_stride = p.row_bytes + 16;
+    const int G = di.sm_count;
+    const int rmax = (ly.K + G - 1) / G + 1;
+    p.rpad = (rmax + 15) & ~15;
+    const size_t fixed = (size_t)p.slot_stride                      /* zero row */
+                         + 2 * kMmaMaxSlots * sizeof(uint64_t) + kMmaWarps * 128 * sizeof(float)
+                         + (size_t)3 * 8 * p.rpad * sizeof(__nv_bfloat16) + 16 + 128;
+    long long slots = ((long long)di.smem_optin - (long long)fixed) / p.slot_stride;
+    if (slots > kMmaMaxSlots) slots = kMmaMaxSlots;
+    if (slots < 17) return COREINFER_ERR_UNSUPPORTED;
+    p.n_slots = (int)slots;
+    const size_t smem = fixed + (size_t)p.n_slots * p.slot_stride;
+    CI_CUDA(cudaMemsetAsync(y, 0, (size_t)batch * d_model * sizeof(float), st));
+    if (gated) {
+        CI_CUDA(cudaFuncSetAttribute(decode_batch_mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        decode_batch_mma_kernel<true><<<G, kMmaBlock, smem, st>>>(p);
+    } else {
+        CI_CUDA(cudaFuncSetAttribute(decode_batch_mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        decode_batch_mma_kernel<false><<<G, kMmaBlock, smem, st>>>(p);
+    }
+    CI_CUDA(cudaGetLastError());
+    return COREINFER_OK;
+}
+
+}  // namespace coreinfer

@@ -53,6 +53,14 @@ def test_small_batches(dtype, gated, B):
     _run_case(B, 72 * (2 if dtype == torch.float32 else 1), 65, gated, dtype, seed=B + 10)
 
 
+@pytest.mark.parametrize("gated", [False, True])
+@pytest.mark.parametrize("B,d,K", [(5, 2048, 20), (8, 4096, 611), (2, 256, 1), (7, 3072, 150), (8, 4096 + 256, 40)])
+def test_batches_on_the_tensor_core_path_and_beside_it(gated, B, d, K):
+    """bf16 rows that are a multiple of 256 columns up to 4096 take the mma kernel (K smaller than
+    the SM count, ragged K, every batch size); 4352 columns fall back to the plain kernels."""
+    _run_case(B, d, K, gated, torch.bfloat16, seed=B * 1000 + K)
+
+
 def test_no_bias_pointers():
     _run_case(1, 512, 100, False, torch.bfloat16, bias=False)
     _run_case(4, 512, 100, True, torch.bfloat16, bias=False)
