@@ -127,6 +127,25 @@ __device__ __forceinline__ void red_add_v4(float* p, float a, float b, float c, 
                  : "memory");
 }
 
+// Bulk reduction shared -> global by the copy engine: adds `bytes` / 4 fp32 values at `src` (shared
+// memory of this CTA, written through the generic proxy and fenced with fence_proxy_async before)
+// into `dst`, element by element, each addition atomic.  Joined to the thread's bulk group.
+__device__ __forceinline__ void fence_proxy_async()
+{
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void bulk_reduce_add_f32(float* dst, uint32_t src, uint32_t bytes)
+{
+    asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f32 [%0], [%1], %2;"
+                 ::"l"(dst), "r"(src), "r"(bytes) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// Returns when every bulk group of this thread has completed (reads and writes).
+__device__ __forceinline__ void bulk_wait_all()
+{
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+
 #endif  // __CUDACC__
 
 }  // namespace coreinfer

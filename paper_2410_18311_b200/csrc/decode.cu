@@ -47,7 +47,7 @@ struct LayerDev {
 
 struct DecodeParams {
     int L, d, nv, row_bytes, slot_bytes, n_slots, rmax;
-    int ysum_ofs;       // shared-memory offset of the two-group hand-over buffer
+    int ysum_ofs;       // shared-memory offset of the buffer holding the CTA's partial y
     const void* x0;
     float* y_last;
     float* y_layers;
@@ -220,7 +220,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
     float* h_s = red + NMAT * kGroupWarps * p.rmax;                 // [rmax]
     float* ss_red = h_s + p.rmax;                                   // [NG][kGroupWarps]
     volatile int* abort_flag = reinterpret_cast<volatile int*>(ss_red + NG * kGroupWarps);
-    float* ysum = reinterpret_cast<float*>(smem + p.ysum_ofs);      // [NG == 2 ? VPT * 256 * EPV : 0]
+    float* ysum = reinterpret_cast<float*>(smem + p.ysum_ofs);      // [VPT * 256 * EPV]: the CTA's partial y
 
     const int tid = threadIdx.x;
     const int G = gridDim.x;
@@ -505,7 +505,12 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
         const bool last = (l == p.L - 1);
         float* ybase = p.ybuf + (size_t)(l % kYBuffers) * kYCopies * d;
         float* ytarget = ybase + (size_t)(cta & (kYCopies - 1)) * d;
-        if (NG == 2) {            // one sum per CTA leaves the chip: group 1 hands its partial to group 0
+        // One sum per CTA leaves the chip, as one bulk reduction: group 1 hands its partial to
+        // group 0 through shared memory, group 0 leaves the CTA's partial there, and the copy
+        // engine adds the whole vector into the target (L2 then sees 128-byte line reductions
+        // instead of a thousand 16-byte atomics per CTA, whose acknowledgements a fence had to
+        // wait for).
+        if (NG == 2) {
             if (grp == 1) {
 #pragma unroll
                 for (int i = 0; i < VPT; ++i)
@@ -519,19 +524,23 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
         if (grp == 0) {
 #pragma unroll
             for (int i = 0; i < VPT; ++i) {
-                const int v = gt + i * kGroupThreads;
-                if (v < nv) {
 #pragma unroll
-                    for (int c = 0; c < PAIRS; c += 2) {
-                        float4 t = make_float4(yacc[i][c].x, yacc[i][c].y, yacc[i][c + 1].x, yacc[i][c + 1].y);
-                        if (NG == 2) {
-                            const float4 o = *reinterpret_cast<const float4*>(ysum + (size_t)v * EPV + 2 * c);
-                            t.x += o.x; t.y += o.y; t.z += o.z; t.w += o.w;
-                        }
-                        red_add_v4(ytarget + (size_t)v * EPV + 2 * c, t.x, t.y, t.z, t.w);
+                for (int c = 0; c < PAIRS; c += 2) {
+                    float4* cell = reinterpret_cast<float4*>(ysum + (size_t)(gt + i * kGroupThreads) * EPV + 2 * c);
+                    float4 t = make_float4(yacc[i][c].x, yacc[i][c].y, yacc[i][c + 1].x, yacc[i][c + 1].y);
+                    if (NG == 2) {
+                        const float4 o = *cell;
+                        t.x += o.x; t.y += o.y; t.z += o.z; t.w += o.w;
                     }
+                    *cell = t;
                 }
             }
+            fence_proxy_async();          // these generic-proxy writes are read by the copy engine next
+        }
+        named_bar_sync(1, NC);
+        if (tid == 0 && !*abort_flag) {
+            bulk_reduce_add_f32(ytarget, smem_u32(ysum), (uint32_t)d * (uint32_t)sizeof(float));
+            bulk_wait_all();
         }
 
         grid_barrier(p.ctrl, (unsigned)(l + 1) * (unsigned)G, abort_flag, NC);
@@ -598,10 +607,11 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
 }
 
 // ------------------------------------------------------------------- host ---
-// fp32 hand-over buffer of the two-group kernels: every thread of a group stores all its columns
+// fp32 buffer in which the CTA's partial y is assembled: every thread of a group stores all its columns
 static size_t ysum_smem_bytes(int groups, int vpt, size_t esize)
 {
-    return groups == 2 ? (size_t)vpt * kGroupThreads * (16 / esize) * sizeof(float) : 0;
+    (void)groups;
+    return (size_t)vpt * kGroupThreads * (16 / esize) * sizeof(float);
 }
 
 static size_t fixed_smem_bytes(int rmax, bool gated, int groups)
