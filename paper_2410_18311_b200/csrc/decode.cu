@@ -47,6 +47,7 @@ struct LayerDev {
 
 struct DecodeParams {
     int L, d, nv, row_bytes, slot_bytes, n_slots, rmax;
+    int runahead;       // ring items of the next layer the producer may request before this layer's exchange is over
     int ysum_ofs;       // shared-memory offset of the buffer holding the CTA's partial y
     const void* x0;
     float* y_last;
@@ -220,6 +221,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
     float* h_s = red + NMAT * kGroupWarps * p.rmax;                 // [rmax]
     float* ss_red = h_s + p.rmax;                                   // [NG][kGroupWarps]
     volatile int* abort_flag = reinterpret_cast<volatile int*>(ss_red + NG * kGroupWarps);
+    volatile int* layers_done = abort_flag + 1;                     // layers whose exchange this CTA has completed
     float* ysum = reinterpret_cast<float*>(smem + p.ysum_ofs);      // [VPT * 256 * EPV]: the CTA's partial y
 
     const int tid = threadIdx.x;
@@ -233,6 +235,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
             mbar_init(smem_u32(&empty_bar[s]), kGroupWarps);     // the warps of the group that reads the slot
         }
         *abort_flag = 0;
+        *layers_done = 0;
         mbar_fence_init();
     }
     __syncthreads();
@@ -257,6 +260,17 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
             for (int q0 = 0; q0 < total; q0 += round_max) {
                 if (*abort_flag) break;
                 const int cnt = min(round_max, total - q0);
+                // Requests of one SM are served in order: while the exchange of the previous layer
+                // is under way, every weight request still queued delays its few small messages
+                // (adds, arrival, poll, read-back) by its own service time.  So only a limited
+                // number of this layer's rows is requested before that exchange is over.
+                if (l > 0 && q0 + cnt > p.runahead) {
+                    const long long t0 = clock64();
+                    while (*layers_done < l && !*abort_flag) {
+                        __nanosleep(64);
+                        if (clock64() - t0 > kWaitCycles) { *abort_flag = 1; atomicMax(p.ctrl, (unsigned)kStatusTimeout); }
+                    }
+                }
                 if (lane < cnt) {
                     const int q = q0 + lane;
                     const uint8_t* src;
@@ -544,6 +558,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
         }
 
         grid_barrier(p.ctrl, (unsigned)(l + 1) * (unsigned)G, abort_flag, NC);
+        if (tid == 0) *layers_done = l + 1;
 
         // ------------------------- next input: (x + y) / rms(x + y), rounded --
         float ss = 0.f;
@@ -755,6 +770,7 @@ static coreinfer_status decode_stack_b1(const coreinfer_layer* layers, int L, co
     if (groups == 2 && slots >= 2 * batch) slots -= slots % (2 * batch);
     p.n_slots = (int)slots;
     const size_t smem = fixed + (size_t)p.n_slots * p.slot_bytes;
+    p.runahead = 16;      // measured at the OPT-6.7B shape: 16 of the 24 slots beats both 8 and no limit
     p.ysum_ofs = (int)((size_t)p.n_slots * p.slot_bytes + fixed0);
     p.x0 = x0;
     p.y_last = y_last;
