@@ -82,9 +82,17 @@ template <> struct Elem<__nv_bfloat16> {
         f[2] = make_float2(__uint_as_float(q.z << 16), __uint_as_float(q.z & 0xffff0000u));
         f[3] = make_float2(__uint_as_float(q.w << 16), __uint_as_float(q.w & 0xffff0000u));
     }
-    static __device__ __forceinline__ float round(float v)
+    // a0 += sum of even-position products, a1 += sum of odd-position products of the 8 bf16
+    // pairs (w, x): mixed-precision FMA, the bf16 product is exact in fp32, one rounding per add
+    static __device__ __forceinline__ void dot(const uint4& w, const uint4& x, float& a0, float& a1)
     {
-        return __bfloat162float(__float2bfloat16_rn(v));
+        const uint32_t ws[4] = {w.x, w.y, w.z, w.w}, xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            asm("{\n\t.reg .b16 wl, wh, xl, xh;\n\t"
+                "mov.b32 {wl, wh}, %2;\n\tmov.b32 {xl, xh}, %3;\n\t"
+                "fma.rn.f32.bf16 %0, wl, xl, %0;\n\tfma.rn.f32.bf16 %1, wh, xh, %1;\n\t}"
+                : "+f"(a0), "+f"(a1) : "r"(ws[c]), "r"(xs[c]));
     }
     static __device__ __forceinline__ uint32_t pack2(float a, float b)
     {
@@ -108,7 +116,13 @@ template <> struct Elem<float> {
         f[0] = make_float2(__uint_as_float(q.x), __uint_as_float(q.y));
         f[1] = make_float2(__uint_as_float(q.z), __uint_as_float(q.w));
     }
-    static __device__ __forceinline__ float round(float v) { return v; }
+    static __device__ __forceinline__ void dot(const uint4& w, const uint4& x, float& a0, float& a1)
+    {
+        a0 = fmaf(__uint_as_float(w.x), __uint_as_float(x.x), a0);
+        a1 = fmaf(__uint_as_float(w.y), __uint_as_float(x.y), a1);
+        a0 = fmaf(__uint_as_float(w.z), __uint_as_float(x.z), a0);
+        a1 = fmaf(__uint_as_float(w.w), __uint_as_float(x.w), a1);
+    }
     static __device__ __forceinline__ uint4 pack(const float2 (&f)[2])
     {
         return make_uint4(__float_as_uint(f[0].x), __float_as_uint(f[0].y), __float_as_uint(f[1].x),
@@ -320,7 +334,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
 
     // this thread's columns: 16-byte vectors gt, gt + 256, ...  vofs[] is clamped so that loads
     // never need a branch (threads beyond the row read vector 0 against a zero x).
-    float2 xr[VPT][PAIRS];
+    uint4 xq[VPT];                // x in the weight type, as loaded
     int vofs[VPT];
 #pragma unroll
     for (int i = 0; i < VPT; ++i) {
@@ -328,7 +342,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
         vofs[i] = (v < nv ? v : 0) * 16;
         uint4 q = make_uint4(0, 0, 0, 0);
         if (v < nv) q = reinterpret_cast<const uint4*>(p.x0)[v];
-        E::unpack(q, xr[i]);
+        xq[i] = q;
         if (p.x_layers && cta == 0 && grp == 0 && v < nv) reinterpret_cast<uint4*>(p.x_layers)[v] = q;
     }
 
@@ -417,15 +431,10 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
                     if (f == own) {               // uniform; keeps part[] statically indexed
 #pragma unroll
                         for (int j = 0; j < BATCH; ++j) {
-                            float2 acc = make_float2(0.f, 0.f);
+                            float a0 = 0.f, a1 = 0.f;
 #pragma unroll
-                            for (int i = 0; i < VPT; ++i) {
-                                float2 w[PAIRS];
-                                E::unpack(q[j][i], w);
-#pragma unroll
-                                for (int c = 0; c < PAIRS; ++c) acc = __ffma2_rn(w[c], xr[i][c], acc);
-                            }
-                            part[f * BATCH + j] = acc.x + acc.y;
+                            for (int i = 0; i < VPT; ++i) E::dot(q[j][i], xq[i], a0, a1);
+                            part[f * BATCH + j] = a0 + a1;
                         }
                     }
                 }
@@ -562,9 +571,11 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
 
         // ------------------------- next input: (x + y) / rms(x + y), rounded --
         float ss = 0.f;
+        float2 xn[VPT][PAIRS];        // x + y in fp32, until the norm is known
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
             const int v = gt + i * kGroupThreads;
+            E::unpack(xq[i], xn[i]);
             if (v < nv) {
 #pragma unroll
                 for (int c = 0; c < PAIRS; c += 2) {
@@ -579,15 +590,15 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
                         if (p.y_layers) *reinterpret_cast<float4*>(p.y_layers + (size_t)l * d + (size_t)v * EPV + 2 * c) = t;
                         if (last) *reinterpret_cast<float4*>(p.y_last + (size_t)v * EPV + 2 * c) = t;
                     }
-                    xr[i][c].x += t.x;
-                    xr[i][c].y += t.y;
-                    xr[i][c + 1].x += t.z;
-                    xr[i][c + 1].y += t.w;
+                    xn[i][c].x += t.x;
+                    xn[i][c].y += t.y;
+                    xn[i][c + 1].x += t.z;
+                    xn[i][c + 1].y += t.w;
                 }
 #pragma unroll
                 for (int c = 0; c < PAIRS; ++c) {
-                    ss = fmaf(xr[i][c].x, xr[i][c].x, ss);
-                    ss = fmaf(xr[i][c].y, xr[i][c].y, ss);
+                    ss = fmaf(xn[i][c].x, xn[i][c].x, ss);
+                    ss = fmaf(xn[i][c].y, xn[i][c].y, ss);
                 }
             }
         }
@@ -611,12 +622,13 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
             const int v = gt + i * kGroupThreads;
 #pragma unroll
             for (int c = 0; c < PAIRS; ++c) {
-                xr[i][c].x = E::round(xr[i][c].x * inv);
-                xr[i][c].y = E::round(xr[i][c].y * inv);
+                xn[i][c].x *= inv;
+                xn[i][c].y *= inv;
             }
+            xq[i] = E::pack(xn[i]);       // rounds to the layer-input type
             if (p.x_layers && cta == (l + 1) % G && grp == 0 && v < nv)
                 reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(p.x_layers) +
-                                         (size_t)(l + 1) * p.row_bytes)[v] = E::pack(xr[i]);
+                                         (size_t)(l + 1) * p.row_bytes)[v] = xq[i];
         }
     }
 }
