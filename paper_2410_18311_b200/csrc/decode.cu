@@ -65,10 +65,11 @@ __host__ __device__ __forceinline__ void slab_of(int cta, int G, int layer, int 
     *k1 = (int)(((long long)(vc + 1) * K) / G);
 }
 
-// items per consumer batch for one group (register budget: 4 * items * vectors per thread)
+// items per consumer batch for one group; a thread holds two batches in registers (the one it
+// computes on and the next one, already loaded): 2 * 4 * items * vectors per thread registers
 __host__ __device__ constexpr int batch_for(int groups, int vpt)
 {
-    return groups == 2 ? 4 : (vpt <= 2 ? 8 : (vpt <= 4 ? 4 : 2));
+    return groups == 2 ? 2 : (vpt <= 2 ? 4 : (vpt <= 4 ? 2 : 1));
 }
 
 // ------------------------------------------------------------ element types --
@@ -225,7 +226,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
     constexpr int NMAT = GATED ? 2 : 1;
     constexpr int NC = NG * kGroupThreads;           // consumer threads
     constexpr int BATCH = batch_for(NG, VPT);        // ring items per batch
-    constexpr int FLUSH = 16 / BATCH;                // own up batches per cross-lane reduction (16 row sums)
+    constexpr int FLUSH = 8 / BATCH;                 // own up batches per cross-lane reduction (8 row sums)
 
     extern __shared__ __align__(128) uint8_t smem[];
     uint8_t* ring = smem;
@@ -405,6 +406,31 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
         skip_n(n);
     };
 
+    // One phase of n_items ring items in batches of BATCH, batch b belonging to group b % NG.  The
+    // group's next batch is pulled into registers before the arithmetic on the current one, so
+    // that the barrier tests and the shared-memory loads of one overlap the arithmetic of the other.
+    auto run_phase = [&](int n_items, auto&& compute) {
+        const int nb = (n_items + BATCH - 1) / BATCH;
+        int at = 0;                               // batch the ring position points at
+        auto count_of = [&](int b) { return min(BATCH, n_items - b * BATCH); };
+        auto seek = [&](int b) { for (; at < b; ++at) skip_n(count_of(at)); };
+        uint4 qa[BATCH][VPT], qb[BATCH][VPT];
+        int b = NG > 1 ? grp : 0;
+        if (b < nb) { seek(b); fetch(qa, count_of(b)); ++at; }
+        while (b < nb) {
+            int bn = b + NG;
+            if (bn < nb) { seek(bn); fetch(qb, count_of(bn)); ++at; }
+            compute(qa, b, count_of(b));
+            b = bn;
+            if (b >= nb) break;
+            bn = b + NG;
+            if (bn < nb) { seek(bn); fetch(qa, count_of(bn)); ++at; }
+            compute(qb, b, count_of(b));
+            b = bn;
+        }
+        seek(nb);
+    };
+
     for (int l = 0; l < p.L; ++l) {
         const LayerDev& ly = p.layers[l];
         int k0, k1;
@@ -414,17 +440,13 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
 
         // ------------------------------------------------ up (+ gate) phase --
         {
-            const int nb = (n_up + BATCH - 1) / BATCH;
-            float part[16];
+            float part[8];
 #pragma unroll
-            for (int j = 0; j < 16; ++j) part[j] = 0.f;
+            for (int j = 0; j < 8; ++j) part[j] = 0.f;
             int own = 0;                          // own batches accumulated in part[]
             int first_b = 0;                      // first of them
-            for (int b = 0; b < nb; ++b) {
-                const int cnt = min(BATCH, n_up - b * BATCH);
-                if (NG > 1 && (b % NG) != grp) { skip_n(cnt); continue; }
-                uint4 q[BATCH][VPT];
-                fetch(q, cnt);
+            const int nb = (n_up + BATCH - 1) / BATCH;
+            run_phase(n_up, [&](const uint4 (&q)[BATCH][VPT], int b, int) {
                 if (own == 0) first_b = b;
 #pragma unroll
                 for (int f = 0; f < FLUSH; ++f) {
@@ -440,28 +462,19 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
                 }
                 ++own;
                 if (own == FLUSH || b + NG >= nb) {
-                    // two independent 8-value reductions (their shuffles interleave)
-                    float lo[8], hi[8];
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) { lo[j] = part[j]; hi[j] = part[8 + j]; }
-                    const float tot_lo = warp_reduce8(lo, lane);
-                    const float tot_hi = warp_reduce8(hi, lane);
+                    const float tot = warp_reduce8(part, lane);
                     if ((lane & 3) == 0) {
-                        const int vi = ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);
-#pragma unroll
-                        for (int half = 0; half < 2; ++half) {
-                            const int pi = half * 8 + vi;                      // index in part[]
-                            const int f = pi / BATCH, j = pi % BATCH;          // own batch f of the window, item j
-                            const int item = (first_b + f * NG) * BATCH + j;   // position in the up phase
-                            if (f < own && item < n_up)
-                                red[((item % NMAT) * kGroupWarps + gw) * p.rmax + item / NMAT] = half ? tot_hi : tot_lo;
-                        }
+                        const int pi = ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);   // index in part[]
+                        const int f = pi / BATCH, j = pi % BATCH;          // own batch f of the window, item j
+                        const int item = (first_b + f * NG) * BATCH + j;   // position in the up phase
+                        if (f < own && item < n_up)
+                            red[((item % NMAT) * kGroupWarps + gw) * p.rmax + item / NMAT] = tot;
                     }
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) part[j] = 0.f;
+                    for (int j = 0; j < 8; ++j) part[j] = 0.f;
                     own = 0;
                 }
-            }
+            });
         }
         named_bar_sync(1, NC);
         for (int r = tid; r < nrows; r += NC) {
@@ -496,29 +509,22 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
                                              E::load1(ly.bdown, v * EPV + 2 * c + 1));
             }
         }
-        {
-            const int nb = (nrows + BATCH - 1) / BATCH;
-            for (int b = 0; b < nb; ++b) {
-                const int cnt = min(BATCH, nrows - b * BATCH);
-                if (NG > 1 && (b % NG) != grp) { skip_n(cnt); continue; }
-                uint4 q[BATCH][VPT];
-                fetch(q, cnt);
+        run_phase(nrows, [&](const uint4 (&q)[BATCH][VPT], int b, int cnt) {
 #pragma unroll
-                for (int j = 0; j < BATCH; ++j) {
-                    const float hk = (j < cnt) ? h_s[b * BATCH + j] : 0.f;
-                    if (hk != 0.f) {                              // uniform: ReLU zeros cost no arithmetic
-                        const float2 hh = make_float2(hk, hk);
+            for (int j = 0; j < BATCH; ++j) {
+                const float hk = (j < cnt) ? h_s[b * BATCH + j] : 0.f;
+                if (hk != 0.f) {                              // uniform: ReLU zeros cost no arithmetic
+                    const float2 hh = make_float2(hk, hk);
 #pragma unroll
-                        for (int i = 0; i < VPT; ++i) {
-                            float2 w[PAIRS];
-                            E::unpack(q[j][i], w);
+                    for (int i = 0; i < VPT; ++i) {
+                        float2 w[PAIRS];
+                        E::unpack(q[j][i], w);
 #pragma unroll
-                            for (int c = 0; c < PAIRS; ++c) yacc[i][c] = __ffma2_rn(w[c], hh, yacc[i][c]);
-                        }
+                        for (int c = 0; c < PAIRS; ++c) yacc[i][c] = __ffma2_rn(w[c], hh, yacc[i][c]);
                     }
                 }
             }
-        }
+        });
 
         // ----------------------------------------- cross-CTA sum of partial y --
         // Every CTA adds its partial into one of kYCopies copies of the layer's target (adds to
