@@ -65,11 +65,10 @@ __host__ __device__ __forceinline__ void slab_of(int cta, int G, int layer, int 
     *k1 = (int)(((long long)(vc + 1) * K) / G);
 }
 
-// items per consumer batch for one group; a thread holds two batches in registers (the one it
-// computes on and the next one, already loaded): 2 * 4 * items * vectors per thread registers
+// items per consumer batch for one group (register budget: 4 * items * vectors per thread)
 __host__ __device__ constexpr int batch_for(int groups, int vpt)
 {
-    return groups == 2 ? 2 : (vpt <= 2 ? 4 : (vpt <= 4 ? 2 : 1));
+    return groups == 2 ? 4 : (vpt <= 2 ? 8 : (vpt <= 4 ? 4 : 2));
 }
 
 // ------------------------------------------------------------ element types --
@@ -83,17 +82,51 @@ template <> struct Elem<__nv_bfloat16> {
         f[2] = make_float2(__uint_as_float(q.z << 16), __uint_as_float(q.z & 0xffff0000u));
         f[3] = make_float2(__uint_as_float(q.w << 16), __uint_as_float(q.w & 0xffff0000u));
     }
-    // a0 += sum of even-position products, a1 += sum of odd-position products of the 8 bf16
-    // pairs (w, x): mixed-precision FMA, the bf16 product is exact in fp32, one rounding per add
-    static __device__ __forceinline__ void dot(const uint4& w, const uint4& x, float& a0, float& a1)
+    // The arithmetic of both phases runs on mma.sync m16n8k16 (bf16 x bf16 products are exact in the
+    // fp32 accumulator).  A thread hands the instruction the very words it loaded: lane = 4 g + t
+    // supplies A[g][2t, 2t+1], A[g+8][2t, 2t+1], A[g][2t+8, 2t+9], A[g+8][2t+8, 2t+9] and
+    // B[2t, 2t+1][g], B[2t+8, 2t+9][g], and receives D[g][2t, 2t+1], D[g+8][2t, 2t+1].
+    static constexpr bool kMma = true;
+    // Up phase, one 16-byte vector of two weight rows a, b against the same vector of x: the A rows
+    // g / g+8 carry this thread's words of row a / row b, B column g carries its words of x, so
+    // D[g][g] (D[g+8][g]) gains the products of the four threads of the quad for row a (row b).
+    static __device__ __forceinline__ void dot2(const uint4& wa, const uint4& wb, const uint4& x, float (&c)[4])
     {
-        const uint32_t ws[4] = {w.x, w.y, w.z, w.w}, xs[4] = {x.x, x.y, x.z, x.w};
+        mma_bf16_16816(c[0], c[1], c[2], c[3], wa.x, wb.x, wa.y, wb.y, x.x, x.y);
+        mma_bf16_16816(c[0], c[1], c[2], c[3], wa.z, wb.z, wa.w, wb.w, x.z, x.w);
+    }
+    // this lane's share of the two row sums: the diagonal entry D[g][g] sits in lane t = g / 2
+    static __device__ __forceinline__ void dot2_result(const float (&c)[4], int lane, float& ra, float& rb)
+    {
+        const int g = lane >> 2, t = lane & 3;
+        const bool mine = (t == (g >> 1));
+        ra = mine ? ((g & 1) ? c[1] : c[0]) : 0.f;
+        rb = mine ? ((g & 1) ? c[3] : c[2]) : 0.f;
+    }
+    // Down phase, y(columns of this vector) += h_a * (row a) + h_b * (row b).  A rows g / g+8 carry
+    // two words of the vector, the k halves carry row a / row b; B[k][n] = h_a for k == n, h_b for
+    // k == n + 8, else 0 (hb.a[], hb.b[]: the three bf16 parts of h_a, h_b, already masked to this
+    // lane's place in that pattern), so D[g][2t + e] gains exactly this thread's own column products.
+    struct HPair { uint32_t a[3], b[3]; float ha, hb; };
+    static __device__ __forceinline__ void axpy2(const uint4& wa, const uint4& wb, const HPair& h, float2 (&y)[4])
+    {
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
-            asm("{\n\t.reg .b16 wl, wh, xl, xh;\n\t"
-                "mov.b32 {wl, wh}, %2;\n\tmov.b32 {xl, xh}, %3;\n\t"
-                "fma.rn.f32.bf16 %0, wl, xl, %0;\n\tfma.rn.f32.bf16 %1, wh, xh, %1;\n\t}"
-                : "+f"(a0), "+f"(a1) : "r"(ws[c]), "r"(xs[c]));
+        for (int s = 0; s < 3; ++s) {
+            mma_bf16_16816(y[0].x, y[0].y, y[1].x, y[1].y, wa.x, wa.y, wb.x, wb.y, h.a[s], h.b[s]);
+            mma_bf16_16816(y[2].x, y[2].y, y[3].x, y[3].y, wa.z, wa.w, wb.z, wb.w, h.a[s], h.b[s]);
+        }
+    }
+    // h -> three bf16 numbers whose sum is h exactly (8 + 8 + 8 significant bits), each one
+    // duplicated into both halves of a word; fourth word: h itself
+    static __device__ __forceinline__ uint4 split_h(float h)
+    {
+        const __nv_bfloat16 p0 = __float2bfloat16_rn(h);
+        const float r1 = h - __bfloat162float(p0);
+        const __nv_bfloat16 p1 = __float2bfloat16_rn(r1);
+        const float r2 = r1 - __bfloat162float(p1);
+        const __nv_bfloat16 p2 = __float2bfloat16_rn(r2);
+        const uint32_t u0 = __bfloat16_as_ushort(p0), u1 = __bfloat16_as_ushort(p1), u2 = __bfloat16_as_ushort(p2);
+        return make_uint4(u0 | (u0 << 16), u1 | (u1 << 16), u2 | (u2 << 16), __float_as_uint(h));
     }
     static __device__ __forceinline__ uint32_t pack2(float a, float b)
     {
@@ -117,13 +150,39 @@ template <> struct Elem<float> {
         f[0] = make_float2(__uint_as_float(q.x), __uint_as_float(q.y));
         f[1] = make_float2(__uint_as_float(q.z), __uint_as_float(q.w));
     }
-    static __device__ __forceinline__ void dot(const uint4& w, const uint4& x, float& a0, float& a1)
+    static constexpr bool kMma = false;
+    // same interface on plain fp32 FMAs: c[0], c[1] two chains of row a, c[2], c[3] of row b
+    static __device__ __forceinline__ void dot2(const uint4& wa, const uint4& wb, const uint4& x, float (&c)[4])
     {
-        a0 = fmaf(__uint_as_float(w.x), __uint_as_float(x.x), a0);
-        a1 = fmaf(__uint_as_float(w.y), __uint_as_float(x.y), a1);
-        a0 = fmaf(__uint_as_float(w.z), __uint_as_float(x.z), a0);
-        a1 = fmaf(__uint_as_float(w.w), __uint_as_float(x.w), a1);
+        c[0] = fmaf(__uint_as_float(wa.x), __uint_as_float(x.x), c[0]);
+        c[1] = fmaf(__uint_as_float(wa.y), __uint_as_float(x.y), c[1]);
+        c[2] = fmaf(__uint_as_float(wb.x), __uint_as_float(x.x), c[2]);
+        c[3] = fmaf(__uint_as_float(wb.y), __uint_as_float(x.y), c[3]);
+        c[0] = fmaf(__uint_as_float(wa.z), __uint_as_float(x.z), c[0]);
+        c[1] = fmaf(__uint_as_float(wa.w), __uint_as_float(x.w), c[1]);
+        c[2] = fmaf(__uint_as_float(wb.z), __uint_as_float(x.z), c[2]);
+        c[3] = fmaf(__uint_as_float(wb.w), __uint_as_float(x.w), c[3]);
     }
+    static __device__ __forceinline__ void dot2_result(const float (&c)[4], int, float& ra, float& rb)
+    {
+        ra = c[0] + c[1];
+        rb = c[2] + c[3];
+    }
+    struct HPair { uint32_t a[3], b[3]; float ha, hb; };
+    static __device__ __forceinline__ void axpy2(const uint4& wa, const uint4& wb, const HPair& h, float2 (&y)[2])
+    {
+        if (h.ha != 0.f) {                            // uniform: ReLU zeros cost no arithmetic
+            const float2 hh = make_float2(h.ha, h.ha);
+            y[0] = __ffma2_rn(make_float2(__uint_as_float(wa.x), __uint_as_float(wa.y)), hh, y[0]);
+            y[1] = __ffma2_rn(make_float2(__uint_as_float(wa.z), __uint_as_float(wa.w)), hh, y[1]);
+        }
+        if (h.hb != 0.f) {
+            const float2 hh = make_float2(h.hb, h.hb);
+            y[0] = __ffma2_rn(make_float2(__uint_as_float(wb.x), __uint_as_float(wb.y)), hh, y[0]);
+            y[1] = __ffma2_rn(make_float2(__uint_as_float(wb.z), __uint_as_float(wb.w)), hh, y[1]);
+        }
+    }
+    static __device__ __forceinline__ uint4 split_h(float h) { return make_uint4(0, 0, 0, __float_as_uint(h)); }
     static __device__ __forceinline__ uint4 pack(const float2 (&f)[2])
     {
         return make_uint4(__float_as_uint(f[0].x), __float_as_uint(f[0].y), __float_as_uint(f[1].x),
@@ -226,15 +285,15 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
     constexpr int NMAT = GATED ? 2 : 1;
     constexpr int NC = NG * kGroupThreads;           // consumer threads
     constexpr int BATCH = batch_for(NG, VPT);        // ring items per batch
-    constexpr int FLUSH = 8 / BATCH;                 // own up batches per cross-lane reduction (8 row sums)
+    constexpr int FLUSH = 16 / BATCH;                // own up batches per cross-lane reduction (16 row sums)
 
     extern __shared__ __align__(128) uint8_t smem[];
     uint8_t* ring = smem;
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(ring + (size_t)p.n_slots * p.slot_bytes);
     uint64_t* empty_bar = full_bar + kMaxSlots;
     float* red = reinterpret_cast<float*>(empty_bar + kMaxSlots);   // [NMAT][kGroupWarps][rmax]
-    float* h_s = red + NMAT * kGroupWarps * p.rmax;                 // [rmax]
-    float* ss_red = h_s + p.rmax;                                   // [NG][kGroupWarps]
+    uint4* h_s = reinterpret_cast<uint4*>(red + NMAT * kGroupWarps * p.rmax);   // [rmax]: parts of h, h
+    float* ss_red = reinterpret_cast<float*>(h_s + p.rmax);         // [NG][kGroupWarps]
     volatile int* abort_flag = reinterpret_cast<volatile int*>(ss_red + NG * kGroupWarps);
     volatile int* layers_done = abort_flag + 1;                     // layers whose exchange this CTA has completed
     float* ysum = reinterpret_cast<float*>(smem + p.ysum_ofs);      // [VPT * 256 * EPV]: the CTA's partial y
@@ -336,17 +395,20 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
     // this thread's columns: 16-byte vectors gt, gt + 256, ...  vofs[] is clamped so that loads
     // never need a branch (threads beyond the row read vector 0 against a zero x).
     uint4 xq[VPT];                // x in the weight type, as loaded
-    int vofs[VPT];
+    uint32_t vofs[VPT];
 #pragma unroll
     for (int i = 0; i < VPT; ++i) {
         const int v = gt + i * kGroupThreads;
-        vofs[i] = (v < nv ? v : 0) * 16;
+        vofs[i] = (uint32_t)(v < nv ? v : 0) * 16u;
         uint4 q = make_uint4(0, 0, 0, 0);
         if (v < nv) q = reinterpret_cast<const uint4*>(p.x0)[v];
         xq[i] = q;
         if (p.x_layers && cta == 0 && grp == 0 && v < nv) reinterpret_cast<uint4*>(p.x_layers)[v] = q;
     }
 
+    // this lane's place in the B operand of the down phase: element k == n of column n = lane / 4
+    const uint32_t hmask = ((lane >> 2) == 2 * (lane & 3)) ? 0x0000ffffu : (((lane >> 2) == 2 * (lane & 3) + 1) ? 0xffff0000u : 0u);
+    const uint32_t ring_s = smem_u32(ring), full_s = smem_u32(full_bar), empty_s = smem_u32(empty_bar);
     int slot = 0;                 // ring position of the next item of the stream
     uint32_t phase = 0;
     auto skip_n = [&](int n) {    // items that belong to the other group
@@ -364,71 +426,35 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
                 int sl = slot + (j < n ? j : 0);
                 uint32_t ph = phase;
                 if (sl >= NS) { sl -= NS; ph ^= 1u; }
-                ready &= mbar_try_wait(smem_u32(&full_bar[sl]), ph);
+                ready &= mbar_try_wait(full_s + 8u * sl, ph);
             }
             if (!ready) {
                 int sl = slot;
                 uint32_t ph = phase;
                 for (int j = 0; j < n; ++j) {
-                    wait_slot(smem_u32(&full_bar[sl]), ph, abort_flag, p.ctrl);
+                    wait_slot(full_s + 8u * sl, ph, abort_flag, p.ctrl);
                     if (++sl == NS) { sl = 0; ph ^= 1u; }
                 }
             }
         }
-        if (n == BATCH) {
 #pragma unroll
-            for (int j = 0; j < BATCH; ++j) {
-                int sl = slot + j;
-                if (sl >= NS) sl -= NS;
-                const uint8_t* row = ring + (size_t)sl * p.slot_bytes;
+        for (int j = 0; j < BATCH; ++j) {
+            int sl = slot + (j < n ? j : 0);
+            if (sl >= NS) sl -= NS;
+            const uint32_t row = ring_s + (uint32_t)sl * (uint32_t)p.slot_bytes;
 #pragma unroll
-                for (int i = 0; i < VPT; ++i) q[j][i] = *reinterpret_cast<const uint4*>(row + vofs[i]);
-            }
-        } else {
-#pragma unroll
-            for (int j = 0; j < BATCH; ++j) {
-                int sl = slot + (j < n ? j : 0);
-                if (sl >= NS) sl -= NS;
-                const uint8_t* row = ring + (size_t)sl * p.slot_bytes;
-#pragma unroll
-                for (int i = 0; i < VPT; ++i) {
-                    q[j][i] = *reinterpret_cast<const uint4*>(row + vofs[i]);
-                    if (j >= n) q[j][i] = make_uint4(0, 0, 0, 0);
-                }
+            for (int i = 0; i < VPT; ++i) {
+                q[j][i] = lds128(row + vofs[i]);
+                if (j >= n) q[j][i] = make_uint4(0, 0, 0, 0);
             }
         }
         __syncwarp();
         if (lane < n && !*abort_flag) {
             int sl = slot + lane;
             if (sl >= NS) sl -= NS;
-            mbar_arrive(smem_u32(&empty_bar[sl]));
+            mbar_arrive(empty_s + 8u * sl);
         }
         skip_n(n);
-    };
-
-    // One phase of n_items ring items in batches of BATCH, batch b belonging to group b % NG.  The
-    // group's next batch is pulled into registers before the arithmetic on the current one, so
-    // that the barrier tests and the shared-memory loads of one overlap the arithmetic of the other.
-    auto run_phase = [&](int n_items, auto&& compute) {
-        const int nb = (n_items + BATCH - 1) / BATCH;
-        int at = 0;                               // batch the ring position points at
-        auto count_of = [&](int b) { return min(BATCH, n_items - b * BATCH); };
-        auto seek = [&](int b) { for (; at < b; ++at) skip_n(count_of(at)); };
-        uint4 qa[BATCH][VPT], qb[BATCH][VPT];
-        int b = NG > 1 ? grp : 0;
-        if (b < nb) { seek(b); fetch(qa, count_of(b)); ++at; }
-        while (b < nb) {
-            int bn = b + NG;
-            if (bn < nb) { seek(bn); fetch(qb, count_of(bn)); ++at; }
-            compute(qa, b, count_of(b));
-            b = bn;
-            if (b >= nb) break;
-            bn = b + NG;
-            if (bn < nb) { seek(bn); fetch(qa, count_of(bn)); ++at; }
-            compute(qb, b, count_of(b));
-            b = bn;
-        }
-        seek(nb);
     };
 
     for (int l = 0; l < p.L; ++l) {
@@ -440,41 +466,54 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
 
         // ------------------------------------------------ up (+ gate) phase --
         {
-            float part[8];
+            const int nb = (n_up + BATCH - 1) / BATCH;
+            float part[16];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) part[j] = 0.f;
+            for (int j = 0; j < 16; ++j) part[j] = 0.f;
             int own = 0;                          // own batches accumulated in part[]
             int first_b = 0;                      // first of them
-            const int nb = (n_up + BATCH - 1) / BATCH;
-            run_phase(n_up, [&](const uint4 (&q)[BATCH][VPT], int b, int) {
+            for (int b = 0; b < nb; ++b) {
+                const int cnt = min(BATCH, n_up - b * BATCH);
+                if (NG > 1 && (b % NG) != grp) { skip_n(cnt); continue; }
+                uint4 q[BATCH][VPT];
+                fetch(q, cnt);
                 if (own == 0) first_b = b;
 #pragma unroll
                 for (int f = 0; f < FLUSH; ++f) {
                     if (f == own) {               // uniform; keeps part[] statically indexed
 #pragma unroll
-                        for (int j = 0; j < BATCH; ++j) {
-                            float a0 = 0.f, a1 = 0.f;
+                        for (int j = 0; j < BATCH; j += 2) {      // two rows at a time
+                            float c[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                            for (int i = 0; i < VPT; ++i) E::dot(q[j][i], xq[i], a0, a1);
-                            part[f * BATCH + j] = a0 + a1;
+                            for (int i = 0; i < VPT; ++i) E::dot2(q[j][i], q[j + 1][i], xq[i], c);
+                            E::dot2_result(c, lane, part[f * BATCH + j], part[f * BATCH + j + 1]);
                         }
                     }
                 }
                 ++own;
                 if (own == FLUSH || b + NG >= nb) {
-                    const float tot = warp_reduce8(part, lane);
+                    // two independent 8-value reductions (their shuffles interleave)
+                    float lo[8], hi[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) { lo[j] = part[j]; hi[j] = part[8 + j]; }
+                    const float tot_lo = warp_reduce8(lo, lane);
+                    const float tot_hi = warp_reduce8(hi, lane);
                     if ((lane & 3) == 0) {
-                        const int pi = ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);   // index in part[]
-                        const int f = pi / BATCH, j = pi % BATCH;          // own batch f of the window, item j
-                        const int item = (first_b + f * NG) * BATCH + j;   // position in the up phase
-                        if (f < own && item < n_up)
-                            red[((item % NMAT) * kGroupWarps + gw) * p.rmax + item / NMAT] = tot;
+                        const int vi = ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);
+#pragma unroll
+                        for (int half = 0; half < 2; ++half) {
+                            const int pi = half * 8 + vi;                      // index in part[]
+                            const int f = pi / BATCH, j = pi % BATCH;          // own batch f of the window, item j
+                            const int item = (first_b + f * NG) * BATCH + j;   // position in the up phase
+                            if (f < own && item < n_up)
+                                red[((item % NMAT) * kGroupWarps + gw) * p.rmax + item / NMAT] = half ? tot_hi : tot_lo;
+                        }
                     }
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) part[j] = 0.f;
+                    for (int j = 0; j < 16; ++j) part[j] = 0.f;
                     own = 0;
                 }
-            });
+            }
         }
         named_bar_sync(1, NC);
         for (int r = tid; r < nrows; r += NC) {
@@ -491,7 +530,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
                 if (ly.bup) u += E::load1(ly.bup, k0 + r);
                 h = fmaxf(u, 0.f);
             }
-            h_s[r] = h;
+            h_s[r] = E::split_h(h);
         }
         named_bar_sync(1, NC);
 
@@ -509,22 +548,30 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
                                              E::load1(ly.bdown, v * EPV + 2 * c + 1));
             }
         }
-        run_phase(nrows, [&](const uint4 (&q)[BATCH][VPT], int b, int cnt) {
+        {
+            const int nb = (nrows + BATCH - 1) / BATCH;
+            for (int b = 0; b < nb; ++b) {
+                const int cnt = min(BATCH, nrows - b * BATCH);
+                if (NG > 1 && (b % NG) != grp) { skip_n(cnt); continue; }
+                uint4 q[BATCH][VPT];
+                fetch(q, cnt);
 #pragma unroll
-            for (int j = 0; j < BATCH; ++j) {
-                const float hk = (j < cnt) ? h_s[b * BATCH + j] : 0.f;
-                if (hk != 0.f) {                              // uniform: ReLU zeros cost no arithmetic
-                    const float2 hh = make_float2(hk, hk);
+                for (int j = 0; j < BATCH; j += 2) {              // two rows at a time
+                    uint4 ha = make_uint4(0, 0, 0, 0), hb = ha;
+                    if (j < cnt) ha = h_s[b * BATCH + j];
+                    if (j + 1 < cnt) hb = h_s[b * BATCH + j + 1];
+                    if (((ha.w | hb.w) & 0x7fffffffu) != 0u) {    // uniform: ReLU zeros cost no arithmetic
+                        typename E::HPair hp;
+                        hp.a[0] = ha.x & hmask; hp.a[1] = ha.y & hmask; hp.a[2] = ha.z & hmask;
+                        hp.b[0] = hb.x & hmask; hp.b[1] = hb.y & hmask; hp.b[2] = hb.z & hmask;
+                        hp.ha = __uint_as_float(ha.w);
+                        hp.hb = __uint_as_float(hb.w);
 #pragma unroll
-                    for (int i = 0; i < VPT; ++i) {
-                        float2 w[PAIRS];
-                        E::unpack(q[j][i], w);
-#pragma unroll
-                        for (int c = 0; c < PAIRS; ++c) yacc[i][c] = __ffma2_rn(w[c], hh, yacc[i][c]);
+                        for (int i = 0; i < VPT; ++i) E::axpy2(q[j][i], q[j + 1][i], hp, yacc[i]);
                     }
                 }
             }
-        });
+        }
 
         // ----------------------------------------- cross-CTA sum of partial y --
         // Every CTA adds its partial into one of kYCopies copies of the layer's target (adds to
@@ -651,7 +698,7 @@ static size_t fixed_smem_bytes(int rmax, bool gated, int groups)
 {
     size_t b = 2 * kMaxSlots * sizeof(uint64_t);
     b += (size_t)(gated ? 2 : 1) * kGroupWarps * rmax * sizeof(float);
-    b += (size_t)rmax * sizeof(float);
+    b += (size_t)rmax * sizeof(uint4);                 // h: three bf16 parts and the value
     b += (size_t)groups * kGroupWarps * sizeof(float) + 16;
     return (b + 127) & ~(size_t)127;
 }
