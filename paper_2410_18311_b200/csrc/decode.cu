@@ -446,14 +446,19 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
             uint32_t ph1 = phase;
             if (s1 >= NS) { s1 -= NS; ph1 ^= 1u; }
             if (cnt < 2) { s1 = s0; ph1 = ph0; }
-            // both barriers are tested back to back (the tests overlap); only if one is not
-            // complete yet fall back to the bounded waits
-            const bool r0 = mbar_try_wait(full_s + 8u * s0, ph0);
-            const bool r1 = mbar_try_wait(full_s + 8u * s1, ph1);
-            if (!(r0 && r1)) {
-                wait_slot(full_s + 8u * s0, ph0, abort_flag, p.ctrl);
-                wait_slot(full_s + 8u * s1, ph1, abort_flag, p.ctrl);
+            // One lane tests for the warp (tests of one barrier by many threads are served one
+            // after the other); both barriers are tested back to back, and only if one is not
+            // complete yet the bounded waits run.  The warp barrier orders the other lanes' loads
+            // after that lane's observation.
+            if (lane == 0) {
+                const bool r0 = mbar_try_wait(full_s + 8u * s0, ph0);
+                const bool r1 = mbar_try_wait(full_s + 8u * s1, ph1);
+                if (!(r0 && r1)) {
+                    wait_slot(full_s + 8u * s0, ph0, abort_flag, p.ctrl);
+                    wait_slot(full_s + 8u * s1, ph1, abort_flag, p.ctrl);
+                }
             }
+            __syncwarp();
             const uint32_t row0 = ring_s + (uint32_t)s0 * (uint32_t)p.slot_bytes;
             const uint32_t row1 = ring_s + (uint32_t)s1 * (uint32_t)p.slot_bytes;
 #pragma unroll
