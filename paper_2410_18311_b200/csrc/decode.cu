@@ -8,31 +8,27 @@
 // so the producer runs ahead across layer boundaries and HBM stays busy while the CTAs exchange
 // partial outputs.
 //
-// Consumers own columns: each of the 512 consumer threads holds the x values of its 16-byte
-// vectors t, t + 512, ... in registers for the whole layer and its partial y likewise.  The
-// ring items of the whole stack form one stream of row pairs (two up rows, or an up and a gate
-// row; later two down rows); every consumer warp walks that stream with a register pipeline a
-// few pairs deep: after the arithmetic on a pair its registers are refilled at once with the
-// pair that many places further down the stream (barrier test, shared-memory loads, slot
-// release), so tests and loads of later pairs overlap the arithmetic of earlier ones, across
-// phase and layer boundaries too: while a layer's partial outputs are exchanged the first pairs
-// of the next layer already sit in registers and their slots are free for the producer.
-// bf16 arithmetic runs on mma.sync: a thread feeds the instruction the very words it loaded.
+// Consumers own columns: thread t of a group holds the x values of its 16-byte vectors
+// t, t + 256, ... in registers for the whole layer and its partial y likewise.  They take ring
+// items in batches: wait for the batch, pull every vector of all its rows into registers with
+// no branch in between (so the loads overlap), free the slots at once, and only then do the
+// arithmetic; slots are held for a few hundred cycles whatever the arithmetic costs.  For rows
+// of at most 8 KB two such groups take alternate batches, so that one group's shared-memory
+// reads overlap the other's arithmetic; wider rows use one group.
 //
-// Exchange per layer: every CTA adds its partial y (d_model fp32) into a global vector with one
-// bulk reduction, then all CTAs meet at a grid barrier, read the full y, and form the next
-// layer's input in registers.  Every wait (slot barriers, grid barrier) is bounded: when one
-// gives up, the CTA marks the workspace status word, stops waiting everywhere, runs the rest of
-// its schedule without synchronising on data, drains its own copies in flight and returns.
+// Exchange per layer: every group adds its partial y (d_model fp32) into a global vector with
+// vector reductions, then all CTAs meet at a grid barrier, read the full y, and every group
+// forms the next layer's input redundantly in registers.  Every wait (slot barriers, grid
+// barrier) is bounded: when one gives up, the CTA marks the workspace status word, stops
+// waiting everywhere, runs the rest of its schedule without synchronising on data, drains its
+// own copies in flight and returns.
 #include "common.cuh"
-#include <stdlib.h>
 
 namespace coreinfer {
 
 constexpr int kMaxSlots = 64;
-constexpr int kConsumers = 512;                        // consumer threads
-constexpr int kConsumerWarps = kConsumers / 32;
-constexpr int kMaxVpt = 4;                             // 16-byte vectors of a row per consumer thread
+constexpr int kGroupThreads = 256;                     // consumer threads per group
+constexpr int kGroupWarps = kGroupThreads / 32;
 constexpr int kCtrlBytes = 256;                        // status word, barrier counter, padding
 constexpr int kYCopies = 2;                            // copies of a reduction target (spreads same-address adds)
 constexpr int kYBuffers = 3;                           // rotating targets: in use, being read, being cleared
@@ -69,8 +65,11 @@ __host__ __device__ __forceinline__ void slab_of(int cta, int G, int layer, int 
     *k1 = (int)(((long long)(vc + 1) * K) / G);
 }
 
-// depth of the consumers' register pipeline in row pairs (2 * 4 * vectors per thread registers each)
-__host__ __device__ constexpr int depth_for(int vpt) { return vpt <= 1 ? 4 : (vpt <= 3 ? 2 : 1); }
+// items per consumer batch for one group (register budget: 4 * items * vectors per thread)
+__host__ __device__ constexpr int batch_for(int groups, int vpt)
+{
+    return groups == 2 ? 4 : (vpt <= 2 ? 8 : (vpt <= 4 ? 4 : 2));
+}
 
 // ------------------------------------------------------------ element types --
 template <typename T> struct Elem;
@@ -83,51 +82,17 @@ template <> struct Elem<__nv_bfloat16> {
         f[2] = make_float2(__uint_as_float(q.z << 16), __uint_as_float(q.z & 0xffff0000u));
         f[3] = make_float2(__uint_as_float(q.w << 16), __uint_as_float(q.w & 0xffff0000u));
     }
-    // The arithmetic of both phases runs on mma.sync m16n8k16 (bf16 x bf16 products are exact in the
-    // fp32 accumulator).  A thread hands the instruction the very words it loaded: lane = 4 g + t
-    // supplies A[g][2t, 2t+1], A[g+8][2t, 2t+1], A[g][2t+8, 2t+9], A[g+8][2t+8, 2t+9] and
-    // B[2t, 2t+1][g], B[2t+8, 2t+9][g], and receives D[g][2t, 2t+1], D[g+8][2t, 2t+1].
-    static constexpr bool kMma = true;
-    // Up phase, one 16-byte vector of two weight rows a, b against the same vector of x: the A rows
-    // g / g+8 carry this thread's words of row a / row b, B column g carries its words of x, so
-    // D[g][g] (D[g+8][g]) gains the products of the four threads of the quad for row a (row b).
-    static __device__ __forceinline__ void dot2(const uint4& wa, const uint4& wb, const uint4& x, float (&c)[4])
+    // a0 += sum of even-position products, a1 += sum of odd-position products of the 8 bf16
+    // pairs (w, x): mixed-precision FMA, the bf16 product is exact in fp32, one rounding per add
+    static __device__ __forceinline__ void dot(const uint4& w, const uint4& x, float& a0, float& a1)
     {
-        mma_bf16_16816(c[0], c[1], c[2], c[3], wa.x, wb.x, wa.y, wb.y, x.x, x.y);
-        mma_bf16_16816(c[0], c[1], c[2], c[3], wa.z, wb.z, wa.w, wb.w, x.z, x.w);
-    }
-    // this lane's share of the two row sums: the diagonal entry D[g][g] sits in lane t = g / 2
-    static __device__ __forceinline__ void dot2_result(const float (&c)[4], int lane, float& ra, float& rb)
-    {
-        const int g = lane >> 2, t = lane & 3;
-        const bool mine = (t == (g >> 1));
-        ra = mine ? ((g & 1) ? c[1] : c[0]) : 0.f;
-        rb = mine ? ((g & 1) ? c[3] : c[2]) : 0.f;
-    }
-    // Down phase, y(columns of this vector) += h_a * (row a) + h_b * (row b).  A rows g / g+8 carry
-    // two words of the vector, the k halves carry row a / row b; B[k][n] = h_a for k == n, h_b for
-    // k == n + 8, else 0 (hb.a[], hb.b[]: the three bf16 parts of h_a, h_b, already masked to this
-    // lane's place in that pattern), so D[g][2t + e] gains exactly this thread's own column products.
-    struct HPair { uint32_t a[3], b[3]; float ha, hb; };
-    static __device__ __forceinline__ void axpy2(const uint4& wa, const uint4& wb, const HPair& h, float2 (&y)[4])
-    {
+        const uint32_t ws[4] = {w.x, w.y, w.z, w.w}, xs[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
-        for (int s = 0; s < 3; ++s) {
-            mma_bf16_16816(y[0].x, y[0].y, y[1].x, y[1].y, wa.x, wa.y, wb.x, wb.y, h.a[s], h.b[s]);
-            mma_bf16_16816(y[2].x, y[2].y, y[3].x, y[3].y, wa.z, wa.w, wb.z, wb.w, h.a[s], h.b[s]);
-        }
-    }
-    // h -> three bf16 numbers whose sum is h exactly (8 + 8 + 8 significant bits), each one
-    // duplicated into both halves of a word; fourth word: h itself
-    static __device__ __forceinline__ uint4 split_h(float h)
-    {
-        const __nv_bfloat16 p0 = __float2bfloat16_rn(h);
-        const float r1 = h - __bfloat162float(p0);
-        const __nv_bfloat16 p1 = __float2bfloat16_rn(r1);
-        const float r2 = r1 - __bfloat162float(p1);
-        const __nv_bfloat16 p2 = __float2bfloat16_rn(r2);
-        const uint32_t u0 = __bfloat16_as_ushort(p0), u1 = __bfloat16_as_ushort(p1), u2 = __bfloat16_as_ushort(p2);
-        return make_uint4(u0 | (u0 << 16), u1 | (u1 << 16), u2 | (u2 << 16), __float_as_uint(h));
+        for (int c = 0; c < 4; ++c)
+            asm("{\n\t.reg .b16 wl, wh, xl, xh;\n\t"
+                "mov.b32 {wl, wh}, %2;\n\tmov.b32 {xl, xh}, %3;\n\t"
+                "fma.rn.f32.bf16 %0, wl, xl, %0;\n\tfma.rn.f32.bf16 %1, wh, xh, %1;\n\t}"
+                : "+f"(a0), "+f"(a1) : "r"(ws[c]), "r"(xs[c]));
     }
     static __device__ __forceinline__ uint32_t pack2(float a, float b)
     {
@@ -151,39 +116,13 @@ template <> struct Elem<float> {
         f[0] = make_float2(__uint_as_float(q.x), __uint_as_float(q.y));
         f[1] = make_float2(__uint_as_float(q.z), __uint_as_float(q.w));
     }
-    static constexpr bool kMma = false;
-    // same interface on plain fp32 FMAs: c[0], c[1] two chains of row a, c[2], c[3] of row b
-    static __device__ __forceinline__ void dot2(const uint4& wa, const uint4& wb, const uint4& x, float (&c)[4])
+    static __device__ __forceinline__ void dot(const uint4& w, const uint4& x, float& a0, float& a1)
     {
-        c[0] = fmaf(__uint_as_float(wa.x), __uint_as_float(x.x), c[0]);
-        c[1] = fmaf(__uint_as_float(wa.y), __uint_as_float(x.y), c[1]);
-        c[2] = fmaf(__uint_as_float(wb.x), __uint_as_float(x.x), c[2]);
-        c[3] = fmaf(__uint_as_float(wb.y), __uint_as_float(x.y), c[3]);
-        c[0] = fmaf(__uint_as_float(wa.z), __uint_as_float(x.z), c[0]);
-        c[1] = fmaf(__uint_as_float(wa.w), __uint_as_float(x.w), c[1]);
-        c[2] = fmaf(__uint_as_float(wb.z), __uint_as_float(x.z), c[2]);
-        c[3] = fmaf(__uint_as_float(wb.w), __uint_as_float(x.w), c[3]);
+        a0 = fmaf(__uint_as_float(w.x), __uint_as_float(x.x), a0);
+        a1 = fmaf(__uint_as_float(w.y), __uint_as_float(x.y), a1);
+        a0 = fmaf(__uint_as_float(w.z), __uint_as_float(x.z), a0);
+        a1 = fmaf(__uint_as_float(w.w), __uint_as_float(x.w), a1);
     }
-    static __device__ __forceinline__ void dot2_result(const float (&c)[4], int, float& ra, float& rb)
-    {
-        ra = c[0] + c[1];
-        rb = c[2] + c[3];
-    }
-    struct HPair { uint32_t a[3], b[3]; float ha, hb; };
-    static __device__ __forceinline__ void axpy2(const uint4& wa, const uint4& wb, const HPair& h, float2 (&y)[2])
-    {
-        if (h.ha != 0.f) {                            // uniform: ReLU zeros cost no arithmetic
-            const float2 hh = make_float2(h.ha, h.ha);
-            y[0] = __ffma2_rn(make_float2(__uint_as_float(wa.x), __uint_as_float(wa.y)), hh, y[0]);
-            y[1] = __ffma2_rn(make_float2(__uint_as_float(wa.z), __uint_as_float(wa.w)), hh, y[1]);
-        }
-        if (h.hb != 0.f) {
-            const float2 hh = make_float2(h.hb, h.hb);
-            y[0] = __ffma2_rn(make_float2(__uint_as_float(wb.x), __uint_as_float(wb.y)), hh, y[0]);
-            y[1] = __ffma2_rn(make_float2(__uint_as_float(wb.z), __uint_as_float(wb.w)), hh, y[1]);
-        }
-    }
-    static __device__ __forceinline__ uint4 split_h(float h) { return make_uint4(0, 0, 0, __float_as_uint(h)); }
     static __device__ __forceinline__ uint4 pack(const float2 (&f)[2])
     {
         return make_uint4(__float_as_uint(f[0].x), __float_as_uint(f[0].y), __float_as_uint(f[1].x),
@@ -274,31 +213,30 @@ __device__ __forceinline__ float warp_reduce8(const float (&v)[8], int lane)
 // ------------------------------------------------------------------- kernel --
 // Ring stream order of one CTA and one layer (producer and consumers walk it in lock step): for
 // each slab row k0 .. k1-1 its up row, then (gated) its gate row; after those, the down rows
-// k0 .. k1-1.  Consumers take the items of a phase two at a time; the pair count of a phase is
-// padded with empty pairs to a multiple of the pipeline depth D, so that every phase starts at
-// pipeline stage 0.
-template <typename T, int VPT, bool GATED>
-__global__ void __launch_bounds__(kConsumers + 32, 1)
+// k0 .. k1-1.  Within each of the two phases the items are cut into batches of BATCH; batch b
+// belongs to consumer group b % NG.
+template <typename T, int NG, int VPT, bool GATED>
+__global__ void __launch_bounds__(NG * kGroupThreads + 32, 1)
 decode_stack_kernel(const __grid_constant__ DecodeParams p)
 {
     using E = Elem<T>;
     constexpr int PAIRS = E::kPairs;
     constexpr int EPV = PAIRS * 2;                   // elements per 16-byte vector
     constexpr int NMAT = GATED ? 2 : 1;
-    constexpr int NC = kConsumers;
-    constexpr int NW = kConsumerWarps;
-    constexpr int D = depth_for(VPT);
+    constexpr int NC = NG * kGroupThreads;           // consumer threads
+    constexpr int BATCH = batch_for(NG, VPT);        // ring items per batch
+    constexpr int FLUSH = 16 / BATCH;                // own up batches per cross-lane reduction (16 row sums)
 
     extern __shared__ __align__(128) uint8_t smem[];
     uint8_t* ring = smem;
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(ring + (size_t)p.n_slots * p.slot_bytes);
     uint64_t* empty_bar = full_bar + kMaxSlots;
-    float* red = reinterpret_cast<float*>(empty_bar + kMaxSlots);   // [NMAT][NW][rmax]
-    uint4* h_s = reinterpret_cast<uint4*>(red + NMAT * NW * p.rmax);   // [rmax]: parts of h, h
-    float* ss_red = reinterpret_cast<float*>(h_s + p.rmax);         // [NW]
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(ss_red + NW);
+    float* red = reinterpret_cast<float*>(empty_bar + kMaxSlots);   // [NMAT][kGroupWarps][rmax]
+    float* h_s = red + NMAT * kGroupWarps * p.rmax;                 // [rmax]
+    float* ss_red = h_s + p.rmax;                                   // [NG][kGroupWarps]
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(ss_red + NG * kGroupWarps);
     volatile int* layers_done = abort_flag + 1;                     // layers whose exchange this CTA has completed
-    float* ysum = reinterpret_cast<float*>(smem + p.ysum_ofs);      // [VPT * NC * EPV]: the CTA's partial y
+    float* ysum = reinterpret_cast<float*>(smem + p.ysum_ofs);      // [VPT * 256 * EPV]: the CTA's partial y
 
     const int tid = threadIdx.x;
     const int G = gridDim.x;
@@ -308,7 +246,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) {
             mbar_init(smem_u32(&full_bar[s]), 1);
-            mbar_init(smem_u32(&empty_bar[s]), NW);              // every consumer warp reads every slot
+            mbar_init(smem_u32(&empty_bar[s]), kGroupWarps);     // the warps of the group that reads the slot
         }
         *abort_flag = 0;
         *layers_done = 0;
@@ -387,99 +325,85 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
     }
 
     // ============================================================ consumers ==
+    const int grp = tid / kGroupThreads;          // consumer group of this thread
+    const int gt = tid % kGroupThreads;           // thread within the group
     const int lane = tid & 31;
-    const int warp = tid >> 5;
+    const int gw = gt >> 5;                       // warp within the group
     const int nv = p.nv;
     const int d = p.d;
 
-    // this thread's columns: 16-byte vectors tid, tid + 512, ...  vofs[] is clamped so that loads
+    // this thread's columns: 16-byte vectors gt, gt + 256, ...  vofs[] is clamped so that loads
     // never need a branch (threads beyond the row read vector 0 against a zero x).
     uint4 xq[VPT];                // x in the weight type, as loaded
-    uint32_t vofs[VPT];
+    int vofs[VPT];
 #pragma unroll
     for (int i = 0; i < VPT; ++i) {
-        const int v = tid + i * NC;
-        vofs[i] = (uint32_t)(v < nv ? v : 0) * 16u;
+        const int v = gt + i * kGroupThreads;
+        vofs[i] = (v < nv ? v : 0) * 16;
         uint4 q = make_uint4(0, 0, 0, 0);
         if (v < nv) q = reinterpret_cast<const uint4*>(p.x0)[v];
         xq[i] = q;
-        if (p.x_layers && cta == 0 && v < nv) reinterpret_cast<uint4*>(p.x_layers)[v] = q;
+        if (p.x_layers && cta == 0 && grp == 0 && v < nv) reinterpret_cast<uint4*>(p.x_layers)[v] = q;
     }
-    // this lane's place in the B operand of the down phase: element k == n of column n = lane / 4
-    const uint32_t hmask = ((lane >> 2) == 2 * (lane & 3)) ? 0x0000ffffu
-                         : (((lane >> 2) == 2 * (lane & 3) + 1) ? 0xffff0000u : 0u);
-    const uint32_t ring_s = smem_u32(ring), full_s = smem_u32(full_bar), empty_s = smem_u32(empty_bar);
 
-    // ---- cursor over the stream of row pairs (all layers), some pairs ahead of the arithmetic
     int slot = 0;                 // ring position of the next item of the stream
     uint32_t phase = 0;
-    int c_layer = 0, c_down = 0;  // layer and phase (0 up, 1 down) the cursor is in
-    int c_pair = 0;               // pair of that phase it points at
-    int c_items, c_pairs;         // items of that phase; its pair count padded to a multiple of D
-    auto items_of = [&](int l, int down) -> int {
-        if (l >= p.L) return 0;
-        int k0, k1;
-        slab_of(cta, G, l, p.layers[l].K, &k0, &k1);
-        return down ? (k1 - k0) : (k1 - k0) * NMAT;
+    auto skip_n = [&](int n) {    // items that belong to the other group
+        slot += n;
+        if (slot >= NS) { slot -= NS; phase ^= 1u; }
     };
-    auto padded_pairs = [&](int items) -> int { return ((items + 1) / 2 + D - 1) / D * D; };
-    c_items = items_of(0, 0);
-    c_pairs = padded_pairs(c_items);
-    // Pull the pair under the cursor into registers (q[0], q[1]: its two rows, zeros where the
-    // pair is short or empty), free its slots, move the cursor on.
-    auto refill = [&](uint4 (&q)[2][VPT]) {
-        while (c_layer < p.L && c_pair >= c_pairs) {             // phase used up (or empty): next one
-            c_pair = 0;
-            if (c_down) { c_down = 0; ++c_layer; } else c_down = 1;
-            c_items = items_of(c_layer, c_down);
-            c_pairs = padded_pairs(c_items);
-        }
-        int cnt = 0;
-        if (c_layer < p.L) {
-            cnt = min(2, max(0, c_items - 2 * c_pair));
-            ++c_pair;
-        }
-        if (cnt > 0) {
-            const int s0 = slot;
-            const uint32_t ph0 = phase;
-            int s1 = slot + 1;
-            uint32_t ph1 = phase;
-            if (s1 >= NS) { s1 -= NS; ph1 ^= 1u; }
-            if (cnt < 2) { s1 = s0; ph1 = ph0; }
-            // One lane tests for the warp (tests of one barrier by many threads are served one
-            // after the other); both barriers are tested back to back, and only if one is not
-            // complete yet the bounded waits run.  The warp barrier orders the other lanes' loads
-            // after that lane's observation.
-            if (lane == 0) {
-                const bool r0 = mbar_try_wait(full_s + 8u * s0, ph0);
-                const bool r1 = mbar_try_wait(full_s + 8u * s1, ph1);
-                if (!(r0 && r1)) {
-                    wait_slot(full_s + 8u * s0, ph0, abort_flag, p.ctrl);
-                    wait_slot(full_s + 8u * s1, ph1, abort_flag, p.ctrl);
+    // wait for the next n items, pull them into registers (q[j][i] = vector i of item j), free them
+    auto fetch = [&](uint4 (&q)[BATCH][VPT], int n) {
+        {
+            // test all barriers of the batch back to back (the tests overlap); only if one is
+            // not complete yet fall back to the bounded waits, one by one
+            bool ready = true;
+#pragma unroll
+            for (int j = 0; j < BATCH; ++j) {
+                int sl = slot + (j < n ? j : 0);
+                uint32_t ph = phase;
+                if (sl >= NS) { sl -= NS; ph ^= 1u; }
+                ready &= mbar_try_wait(smem_u32(&full_bar[sl]), ph);
+            }
+            if (!ready) {
+                int sl = slot;
+                uint32_t ph = phase;
+                for (int j = 0; j < n; ++j) {
+                    wait_slot(smem_u32(&full_bar[sl]), ph, abort_flag, p.ctrl);
+                    if (++sl == NS) { sl = 0; ph ^= 1u; }
                 }
             }
-            __syncwarp();
-            const uint32_t row0 = ring_s + (uint32_t)s0 * (uint32_t)p.slot_bytes;
-            const uint32_t row1 = ring_s + (uint32_t)s1 * (uint32_t)p.slot_bytes;
+        }
+        if (n == BATCH) {
 #pragma unroll
-            for (int i = 0; i < VPT; ++i) {
-                q[0][i] = lds128(row0 + vofs[i]);
-                q[1][i] = lds128(row1 + vofs[i]);
-                if (cnt < 2) q[1][i] = make_uint4(0, 0, 0, 0);
+            for (int j = 0; j < BATCH; ++j) {
+                int sl = slot + j;
+                if (sl >= NS) sl -= NS;
+                const uint8_t* row = ring + (size_t)sl * p.slot_bytes;
+#pragma unroll
+                for (int i = 0; i < VPT; ++i) q[j][i] = *reinterpret_cast<const uint4*>(row + vofs[i]);
             }
-            __syncwarp();
-            if (lane < cnt) mbar_arrive(empty_s + 8u * (lane == 0 ? s0 : s1));
-            slot += cnt;
-            if (slot >= NS) { slot -= NS; phase ^= 1u; }
         } else {
 #pragma unroll
-            for (int i = 0; i < VPT; ++i) q[0][i] = q[1][i] = make_uint4(0, 0, 0, 0);
-        }
-    };
-
-    uint4 q[D][2][VPT];           // pipeline stages: stage s holds pair (s mod D) of the next D pairs
+            for (int j = 0; j < BATCH; ++j) {
+                int sl = slot + (j < n ? j : 0);
+                if (sl >= NS) sl -= NS;
+                const uint8_t* row = ring + (size_t)sl * p.slot_bytes;
 #pragma unroll
-    for (int s = 0; s < D; ++s) refill(q[s]);
+                for (int i = 0; i < VPT; ++i) {
+                    q[j][i] = *reinterpret_cast<const uint4*>(row + vofs[i]);
+                    if (j >= n) q[j][i] = make_uint4(0, 0, 0, 0);
+                }
+            }
+        }
+        __syncwarp();
+        if (lane < n && !*abort_flag) {
+            int sl = slot + lane;
+            if (sl >= NS) sl -= NS;
+            mbar_arrive(smem_u32(&empty_bar[sl]));
+        }
+        skip_n(n);
+    };
 
     for (int l = 0; l < p.L; ++l) {
         const LayerDev& ly = p.layers[l];
@@ -489,43 +413,72 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
         const int n_up = nrows * NMAT;
 
         // ------------------------------------------------ up (+ gate) phase --
-        for (int i0 = 0, np = padded_pairs(n_up); i0 < np; i0 += D) {
-            float part[8];
+        {
+            const int nb = (n_up + BATCH - 1) / BATCH;
+            float part[16];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) part[j] = 0.f;
+            for (int j = 0; j < 16; ++j) part[j] = 0.f;
+            int own = 0;                          // own batches accumulated in part[]
+            int first_b = 0;                      // first of them
+            for (int b = 0; b < nb; ++b) {
+                const int cnt = min(BATCH, n_up - b * BATCH);
+                if (NG > 1 && (b % NG) != grp) { skip_n(cnt); continue; }
+                uint4 q[BATCH][VPT];
+                fetch(q, cnt);
+                if (own == 0) first_b = b;
 #pragma unroll
-            for (int s = 0; s < D; ++s) {
-                float c[4] = {0.f, 0.f, 0.f, 0.f};
+                for (int f = 0; f < FLUSH; ++f) {
+                    if (f == own) {               // uniform; keeps part[] statically indexed
 #pragma unroll
-                for (int i = 0; i < VPT; ++i) E::dot2(q[s][0][i], q[s][1][i], xq[i], c);
-                E::dot2_result(c, lane, part[2 * s], part[2 * s + 1]);
-                refill(q[s]);
-            }
-            // the 2 D item sums of this trip, summed over the warp
-            const float tot = warp_reduce8(part, lane);
-            if ((lane & 3) == 0) {
-                const int vi = ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);   // index in part[]
-                const int item = 2 * i0 + vi;                                                       // position in the phase
-                if (vi < 2 * D && item < n_up)
-                    red[((item % NMAT) * NW + warp) * p.rmax + item / NMAT] = tot;
+                        for (int j = 0; j < BATCH; ++j) {
+                            float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+                            for (int i = 0; i < VPT; ++i) E::dot(q[j][i], xq[i], a0, a1);
+                            part[f * BATCH + j] = a0 + a1;
+                        }
+                    }
+                }
+                ++own;
+                if (own == FLUSH || b + NG >= nb) {
+                    // two independent 8-value reductions (their shuffles interleave)
+                    float lo[8], hi[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) { lo[j] = part[j]; hi[j] = part[8 + j]; }
+                    const float tot_lo = warp_reduce8(lo, lane);
+                    const float tot_hi = warp_reduce8(hi, lane);
+                    if ((lane & 3) == 0) {
+                        const int vi = ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);
+#pragma unroll
+                        for (int half = 0; half < 2; ++half) {
+                            const int pi = half * 8 + vi;                      // index in part[]
+                            const int f = pi / BATCH, j = pi % BATCH;          // own batch f of the window, item j
+                            const int item = (first_b + f * NG) * BATCH + j;   // position in the up phase
+                            if (f < own && item < n_up)
+                                red[((item % NMAT) * kGroupWarps + gw) * p.rmax + item / NMAT] = half ? tot_hi : tot_lo;
+                        }
+                    }
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) part[j] = 0.f;
+                    own = 0;
+                }
             }
         }
         named_bar_sync(1, NC);
         for (int r = tid; r < nrows; r += NC) {
             float u = 0.f;
 #pragma unroll
-            for (int w = 0; w < NW; ++w) u += red[w * p.rmax + r];
+            for (int w = 0; w < kGroupWarps; ++w) u += red[w * p.rmax + r];
             float h;
             if (GATED) {
                 float g = 0.f;
 #pragma unroll
-                for (int w = 0; w < NW; ++w) g += red[(NW + w) * p.rmax + r];
+                for (int w = 0; w < kGroupWarps; ++w) g += red[(kGroupWarps + w) * p.rmax + r];
                 h = fmaxf(g, 0.f) * u;
             } else {
                 if (ly.bup) u += E::load1(ly.bup, k0 + r);
                 h = fmaxf(u, 0.f);
             }
-            h_s[r] = E::split_h(h);
+            h_s[r] = h;
         }
         named_bar_sync(1, NC);
 
@@ -533,33 +486,37 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
         float2 yacc[VPT][PAIRS];
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
-            const int v = tid + i * NC;
+            const int v = gt + i * kGroupThreads;
 #pragma unroll
             for (int c = 0; c < PAIRS; ++c) yacc[i][c] = make_float2(0.f, 0.f);
-            if (cta == 0 && ly.bdown && v < nv) {               // the bias enters the sum exactly once
+            if (cta == 0 && grp == 0 && ly.bdown && v < nv) {   // the bias enters the sum exactly once
 #pragma unroll
                 for (int c = 0; c < PAIRS; ++c)
                     yacc[i][c] = make_float2(E::load1(ly.bdown, v * EPV + 2 * c),
                                              E::load1(ly.bdown, v * EPV + 2 * c + 1));
             }
         }
-        for (int i0 = 0, np = padded_pairs(nrows); i0 < np; i0 += D) {
+        {
+            const int nb = (nrows + BATCH - 1) / BATCH;
+            for (int b = 0; b < nb; ++b) {
+                const int cnt = min(BATCH, nrows - b * BATCH);
+                if (NG > 1 && (b % NG) != grp) { skip_n(cnt); continue; }
+                uint4 q[BATCH][VPT];
+                fetch(q, cnt);
 #pragma unroll
-            for (int s = 0; s < D; ++s) {
-                const int r = 2 * (i0 + s);
-                uint4 ha = make_uint4(0, 0, 0, 0), hb = ha;
-                if (r < nrows) ha = h_s[r];
-                if (r + 1 < nrows) hb = h_s[r + 1];
-                if (((ha.w | hb.w) & 0x7fffffffu) != 0u) {      // uniform: ReLU zeros cost no arithmetic
-                    typename E::HPair hp;
-                    hp.a[0] = ha.x & hmask; hp.a[1] = ha.y & hmask; hp.a[2] = ha.z & hmask;
-                    hp.b[0] = hb.x & hmask; hp.b[1] = hb.y & hmask; hp.b[2] = hb.z & hmask;
-                    hp.ha = __uint_as_float(ha.w);
-                    hp.hb = __uint_as_float(hb.w);
+                for (int j = 0; j < BATCH; ++j) {
+                    const float hk = (j < cnt) ? h_s[b * BATCH + j] : 0.f;
+                    if (hk != 0.f) {                              // uniform: ReLU zeros cost no arithmetic
+                        const float2 hh = make_float2(hk, hk);
 #pragma unroll
-                    for (int i = 0; i < VPT; ++i) E::axpy2(q[s][0][i], q[s][1][i], hp, yacc[i]);
+                        for (int i = 0; i < VPT; ++i) {
+                            float2 w[PAIRS];
+                            E::unpack(q[j][i], w);
+#pragma unroll
+                            for (int c = 0; c < PAIRS; ++c) yacc[i][c] = __ffma2_rn(w[c], hh, yacc[i][c]);
+                        }
+                    }
                 }
-                refill(q[s]);
             }
         }
 
@@ -568,19 +525,41 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
         // one address are serialised in L2, so they are spread); after the grid barrier every
         // thread sums the copies for its columns.  Targets rotate over three buffers: while layer
         // l's is read, the one layer l+2 will use is cleared (last read before the barrier of l).
-        // The partial leaves the CTA as one bulk reduction from shared memory: the copy engine
-        // adds the whole vector into the target (L2 then sees 128-byte line reductions instead of
-        // a thousand 16-byte atomics per CTA, whose acknowledgements a fence had to wait for).
         const bool last = (l == p.L - 1);
         float* ybase = p.ybuf + (size_t)(l % kYBuffers) * kYCopies * d;
         float* ytarget = ybase + (size_t)(cta & (kYCopies - 1)) * d;
+        // One sum per CTA leaves the chip, as one bulk reduction: group 1 hands its partial to
+        // group 0 through shared memory, group 0 leaves the CTA's partial there, and the copy
+        // engine adds the whole vector into the target (L2 then sees 128-byte line reductions
+        // instead of a thousand 16-byte atomics per CTA, whose acknowledgements a fence had to
+        // wait for).
+        if (NG == 2) {
+            if (grp == 1) {
 #pragma unroll
-        for (int i = 0; i < VPT; ++i)
+                for (int i = 0; i < VPT; ++i)
 #pragma unroll
-            for (int c = 0; c < PAIRS; c += 2)
-                *reinterpret_cast<float4*>(ysum + (size_t)(tid + i * NC) * EPV + 2 * c) =
-                    make_float4(yacc[i][c].x, yacc[i][c].y, yacc[i][c + 1].x, yacc[i][c + 1].y);
-        fence_proxy_async();              // these generic-proxy writes are read by the copy engine next
+                    for (int c = 0; c < PAIRS; c += 2)
+                        *reinterpret_cast<float4*>(ysum + (size_t)(gt + i * kGroupThreads) * EPV + 2 * c) =
+                            make_float4(yacc[i][c].x, yacc[i][c].y, yacc[i][c + 1].x, yacc[i][c + 1].y);
+            }
+            named_bar_sync(1, NC);
+        }
+        if (grp == 0) {
+#pragma unroll
+            for (int i = 0; i < VPT; ++i) {
+#pragma unroll
+                for (int c = 0; c < PAIRS; c += 2) {
+                    float4* cell = reinterpret_cast<float4*>(ysum + (size_t)(gt + i * kGroupThreads) * EPV + 2 * c);
+                    float4 t = make_float4(yacc[i][c].x, yacc[i][c].y, yacc[i][c + 1].x, yacc[i][c + 1].y);
+                    if (NG == 2) {
+                        const float4 o = *cell;
+                        t.x += o.x; t.y += o.y; t.z += o.z; t.w += o.w;
+                    }
+                    *cell = t;
+                }
+            }
+            fence_proxy_async();          // these generic-proxy writes are read by the copy engine next
+        }
         named_bar_sync(1, NC);
         if (tid == 0 && !*abort_flag) {
             bulk_reduce_add_f32(ytarget, smem_u32(ysum), (uint32_t)d * (uint32_t)sizeof(float));
@@ -595,7 +574,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
         float2 xn[VPT][PAIRS];        // x + y in fp32, until the norm is known
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
-            const int v = tid + i * NC;
+            const int v = gt + i * kGroupThreads;
             E::unpack(xq[i], xn[i]);
             if (v < nv) {
 #pragma unroll
@@ -607,7 +586,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
                     float4 t = u[0];
 #pragma unroll
                     for (int cp = 1; cp < kYCopies; ++cp) { t.x += u[cp].x; t.y += u[cp].y; t.z += u[cp].z; t.w += u[cp].w; }
-                    if (cta == l % G) {
+                    if (cta == l % G && grp == 0) {
                         if (p.y_layers) *reinterpret_cast<float4*>(p.y_layers + (size_t)l * d + (size_t)v * EPV + 2 * c) = t;
                         if (last) *reinterpret_cast<float4*>(p.y_last + (size_t)v * EPV + 2 * c) = t;
                     }
@@ -629,24 +608,25 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
             for (int i = cta * NC + tid; i < n4; i += G * NC) z[i] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
         if (last) break;
+        // every group holds all columns, so each forms the norm on its own (same sums, same order)
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-        if (lane == 0) ss_red[warp] = ss;
-        named_bar_sync(1, NC);
+        if (lane == 0) ss_red[grp * kGroupWarps + gw] = ss;
+        named_bar_sync(2 + grp, kGroupThreads);
         float tot = 0.f;
 #pragma unroll
-        for (int w = 0; w < NW; ++w) tot += ss_red[w];
+        for (int w = 0; w < kGroupWarps; ++w) tot += ss_red[grp * kGroupWarps + w];
         const float inv = 1.0f / sqrtf(tot / (float)d);
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
-            const int v = tid + i * NC;
+            const int v = gt + i * kGroupThreads;
 #pragma unroll
             for (int c = 0; c < PAIRS; ++c) {
                 xn[i][c].x *= inv;
                 xn[i][c].y *= inv;
             }
             xq[i] = E::pack(xn[i]);       // rounds to the layer-input type
-            if (p.x_layers && cta == (l + 1) % G && v < nv)
+            if (p.x_layers && cta == (l + 1) % G && grp == 0 && v < nv)
                 reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(p.x_layers) +
                                          (size_t)(l + 1) * p.row_bytes)[v] = xq[i];
         }
@@ -654,25 +634,26 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
 }
 
 // ------------------------------------------------------------------- host ---
-// fp32 buffer in which the CTA's partial y is assembled: every consumer thread stores all its columns
-static size_t ysum_smem_bytes(int vpt, size_t esize)
+// fp32 buffer in which the CTA's partial y is assembled: every thread of a group stores all its columns
+static size_t ysum_smem_bytes(int groups, int vpt, size_t esize)
 {
-    return (size_t)vpt * kConsumers * (16 / esize) * sizeof(float);
+    (void)groups;
+    return (size_t)vpt * kGroupThreads * (16 / esize) * sizeof(float);
 }
 
-static size_t fixed_smem_bytes(int rmax, bool gated)
+static size_t fixed_smem_bytes(int rmax, bool gated, int groups)
 {
     size_t b = 2 * kMaxSlots * sizeof(uint64_t);
-    b += (size_t)(gated ? 2 : 1) * kConsumerWarps * rmax * sizeof(float);
-    b += (size_t)rmax * sizeof(uint4);                 // h: three bf16 parts and the value
-    b += (size_t)kConsumerWarps * sizeof(float) + 16;
+    b += (size_t)(gated ? 2 : 1) * kGroupWarps * rmax * sizeof(float);
+    b += (size_t)rmax * sizeof(float);
+    b += (size_t)groups * kGroupWarps * sizeof(float) + 16;
     return (b + 127) & ~(size_t)127;
 }
 
-template <typename T, int VPT, bool GATED>
+template <typename T, int NG, int VPT, bool GATED>
 static coreinfer_status launch_one(const DecodeParams& p, int grid, size_t smem, cudaStream_t st)
 {
-    auto kern = decode_stack_kernel<T, VPT, GATED>;
+    auto kern = decode_stack_kernel<T, NG, VPT, GATED>;
     static thread_local size_t configured[64] = {0};
     int dev = 0;
     CI_CUDA(cudaGetDevice(&dev));
@@ -682,7 +663,7 @@ static coreinfer_status launch_one(const DecodeParams& p, int grid, size_t smem,
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3((unsigned)(kConsumers + 32));
+    cfg.blockDim = dim3((unsigned)(NG * kGroupThreads + 32));
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -694,15 +675,24 @@ static coreinfer_status launch_one(const DecodeParams& p, int grid, size_t smem,
     return COREINFER_OK;
 }
 
-template <typename T, bool GATED>
-static coreinfer_status launch_shape(int vpt, const DecodeParams& p, int grid, size_t smem, cudaStream_t st)
+static int groups_for(int nv) { return nv <= 2 * kGroupThreads ? 2 : 1; }
+static int vpt_for(int nv)
 {
-    switch (vpt) {
-    case 1: return launch_one<T, 1, GATED>(p, grid, smem, st);
-    case 2: return launch_one<T, 2, GATED>(p, grid, smem, st);
-    case 3: return launch_one<T, 3, GATED>(p, grid, smem, st);
-    default: return launch_one<T, 4, GATED>(p, grid, smem, st);
+    const int v = (nv + kGroupThreads - 1) / kGroupThreads;
+    return v <= 1 ? 1 : v <= 2 ? 2 : v <= 3 ? 3 : v <= 5 ? 5 : 8;
+}
+
+template <typename T, bool GATED>
+static coreinfer_status launch_shape(int groups, int vpt, const DecodeParams& p, int grid, size_t smem,
+                                     cudaStream_t st)
+{
+    if (groups == 2) {
+        if (vpt <= 1) return launch_one<T, 2, 1, GATED>(p, grid, smem, st);
+        return launch_one<T, 2, 2, GATED>(p, grid, smem, st);
     }
+    if (vpt <= 3) return launch_one<T, 1, 3, GATED>(p, grid, smem, st);
+    if (vpt <= 5) return launch_one<T, 1, 5, GATED>(p, grid, smem, st);
+    return launch_one<T, 1, 8, GATED>(p, grid, smem, st);
 }
 
 static coreinfer_status check_common(const void* x, int batch, coreinfer_dtype dtype,
@@ -775,19 +765,24 @@ static coreinfer_status decode_stack_b1(const coreinfer_layer* layers, int L, co
         if (layers[l].K > Kmax) Kmax = layers[l].K;
     }
     p.rmax = (Kmax + G - 1) / G + 1;
-    const int vpt = (p.nv + kConsumers - 1) / kConsumers;
-    if (vpt > kMaxVpt)
+    const int groups = groups_for(p.nv);
+    if ((p.nv + kGroupThreads - 1) / kGroupThreads > 8)
         CI_FAIL(COREINFER_ERR_UNSUPPORTED, "d_model %d is too wide for this kernel (max %d bytes per row)",
-                d_model, kMaxVpt * kConsumers * 16);
-    const size_t fixed0 = fixed_smem_bytes(p.rmax, gated);
-    const size_t fixed = fixed0 + ysum_smem_bytes(vpt, esize);
-    if (fixed + 4 * (size_t)p.slot_bytes > (size_t)di.smem_optin)
+                d_model, 8 * kGroupThreads * 16);
+    const int vpt = groups == 2 ? ((p.nv + kGroupThreads - 1) / kGroupThreads <= 1 ? 1 : 2) : vpt_for(p.nv);
+    const int batch = batch_for(groups, groups == 2 ? vpt : (vpt <= 3 ? 3 : vpt));
+    const size_t fixed0 = fixed_smem_bytes(p.rmax, gated, groups);
+    const size_t fixed = fixed0 + ysum_smem_bytes(groups, vpt, esize);
+    if (fixed + (size_t)batch * p.slot_bytes > (size_t)di.smem_optin)
         CI_FAIL(COREINFER_ERR_UNSUPPORTED, "K = %d, d_model = %d do not fit in shared memory", Kmax, d_model);
     long long slots = ((long long)di.smem_optin - (long long)fixed) / p.slot_bytes;
     if (slots > kMaxSlots) slots = kMaxSlots;
+    // With two groups a slot must always come back to the same group (a group never waits on the
+    // other's items, so only then can it never be a full ring pass ahead of a barrier it tests).
+    if (groups == 2 && slots >= 2 * batch) slots -= slots % (2 * batch);
     p.n_slots = (int)slots;
     const size_t smem = fixed + (size_t)p.n_slots * p.slot_bytes;
-    { const char* e = getenv("CI_DEV_RUNAHEAD"); p.runahead = e ? atoi(e) : 16; }
+    p.runahead = 16;      // measured at the OPT-6.7B shape: 16 of the 24 slots beats both 8 and no limit
     p.ysum_ofs = (int)((size_t)p.n_slots * p.slot_bytes + fixed0);
     p.x0 = x0;
     p.y_last = y_last;
@@ -799,10 +794,10 @@ static coreinfer_status decode_stack_b1(const coreinfer_layer* layers, int L, co
     // Control words and the reduction targets start at zero.
     CI_CUDA(cudaMemsetAsync(workspace, 0, b1_workspace_bytes(d_model), st));
     if (dtype == COREINFER_BF16)
-        return gated ? launch_shape<__nv_bfloat16, true>(vpt, p, G, smem, st)
-                     : launch_shape<__nv_bfloat16, false>(vpt, p, G, smem, st);
-    return gated ? launch_shape<float, true>(vpt, p, G, smem, st)
-                 : launch_shape<float, false>(vpt, p, G, smem, st);
+        return gated ? launch_shape<__nv_bfloat16, true>(groups, vpt, p, G, smem, st)
+                     : launch_shape<__nv_bfloat16, false>(groups, vpt, p, G, smem, st);
+    return gated ? launch_shape<float, true>(groups, vpt, p, G, smem, st)
+                 : launch_shape<float, false>(groups, vpt, p, G, smem, st);
 }
 
 // decode_batch.cu
