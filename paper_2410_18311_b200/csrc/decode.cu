@@ -271,18 +271,22 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
             const int n = k1 - k0;
             const int n_up = n * NMAT;            // items of the up (+ gate) phase
             const int total = n_up + n;           // + the down rows
-            for (int q0 = 0; q0 < total; q0 += round_max) {
+            for (int q0 = 0, cnt = 0; q0 < total; q0 += cnt) {
                 if (*abort_flag) break;
-                const int cnt = min(round_max, total - q0);
-                // Requests of one SM are served in order: while the exchange of the previous layer
-                // is under way, every weight request still queued delays its few small messages
-                // (adds, arrival, poll, read-back) by its own service time.  So only a limited
-                // number of this layer's rows is requested before that exchange is over.
-                if (l > 0 && q0 + cnt > p.runahead) {
-                    const long long t0 = clock64();
-                    while (*layers_done < l && !*abort_flag) {
-                        __nanosleep(64);
-                        if (clock64() - t0 > kWaitCycles) { *abort_flag = 1; atomicMax(p.ctrl, (unsigned)kStatusTimeout); }
+                cnt = min(round_max, total - q0);
+                // Every weight request in flight delays the few small messages of the previous
+                // layer's exchange (adds, arrival, poll, read-back), which queue behind it.  So
+                // only a limited number of this layer's rows is requested before that exchange is
+                // over: a round is cut at the limit, and beyond it the producer waits.
+                if (l > 0 && q0 + cnt > p.runahead && *layers_done < l) {
+                    if (q0 < p.runahead) {
+                        cnt = p.runahead - q0;
+                    } else {
+                        const long long t0 = clock64();
+                        while (*layers_done < l && !*abort_flag) {
+                            __nanosleep(64);
+                            if (clock64() - t0 > kWaitCycles) { *abort_flag = 1; atomicMax(p.ctrl, (unsigned)kStatusTimeout); }
+                        }
                     }
                 }
                 if (lane < cnt) {
@@ -567,7 +571,6 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
         }
 
         grid_barrier(p.ctrl, (unsigned)(l + 1) * (unsigned)G, abort_flag, NC);
-        if (tid == 0) *layers_done = l + 1;
 
         // ------------------------- next input: (x + y) / rms(x + y), rounded --
         float ss = 0.f;
@@ -613,6 +616,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
         for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
         if (lane == 0) ss_red[grp * kGroupWarps + gw] = ss;
         named_bar_sync(2 + grp, kGroupThreads);
+        if (tid == 0) *layers_done = l + 1;       // group 0 has read the sum: the producer may go on
         float tot = 0.f;
 #pragma unroll
         for (int w = 0; w < kGroupWarps; ++w) tot += ss_red[grp * kGroupWarps + w];
