@@ -191,13 +191,13 @@ coreinfer_status coreinfer_ffn_decode_stack(const coreinfer_layer* layers, int32
  * left to carve a workspace from; code running under a host framework that forbids cudaMalloc
  * on its threads, since that call synchronises the device; a latency-critical loop that may
  * not call an allocator.  The kernel's scratch (control words and per-layer reduction targets)
- * sits in a fixed 256 KiB array inside the library image, so every GPU that loads the library
- * gives up 256 KiB for the life of the process, and the call itself allocates nothing (no
+ * sits in a fixed 128 KiB array inside the library image, so every GPU that loads the library
+ * gives up 128 KiB for the life of the process, and the call itself allocates nothing (no
  * cudaMalloc / cudaFree, no allocating library routine).
  *
  * Arguments and results are those of coreinfer_ffn_decode_stack without the workspace pair.
- * Limit: the scratch the kernel needs, 256 + 24 * d_model bytes (any number of layers), must fit
- * in 256 KiB, i.e. d_model <= 10912; wider models return COREINFER_ERR_UNSUPPORTED and enqueue
+ * Limit: the scratch the kernel needs, 256 + 12 * d_model bytes (any number of layers), must fit
+ * in 128 KiB, i.e. d_model <= 10901; wider models return COREINFER_ERR_UNSUPPORTED and enqueue
  * nothing -- use the workspace variant for them.
  * The first call on each device looks up the array's device address (cudaGetSymbolAddress),
  * which is set-up work rather than stream work: make that first call before starting any

@@ -193,7 +193,7 @@ def coreinfer_ffn_decode_stack(layers, x0, kind, y_last, y_layers, x_layers, wor
 
 def coreinfer_ffn_decode_stack_noalloc(layers, x0, kind, y_last, y_layers, x_layers, stream=None):
     """coreinfer_ffn_decode_stack for callers that cannot allocate: no workspace argument, the
-    scratch is a fixed 256 KiB array inside the library (d_model beyond 10912 raises ERR_UNSUPPORTED).
+    scratch is a fixed 128 KiB array inside the library (d_model beyond 10901 raises ERR_UNSUPPORTED).
     Calls that may overlap on the GPU must not share it; make the first call on a device
     outside stream capture."""
     batch, d_model = x0.shape

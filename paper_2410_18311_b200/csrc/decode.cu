@@ -30,7 +30,7 @@ constexpr int kMaxSlots = 64;
 constexpr int kGroupThreads = 256;                     // consumer threads per group
 constexpr int kGroupWarps = kGroupThreads / 32;
 constexpr int kCtrlBytes = 256;                        // status word, barrier counter, padding
-constexpr int kYCopies = 2;                            // copies of a reduction target (spreads same-address adds)
+constexpr int kYCopies = 1;                            // copies of a reduction target (more spread same-address adds, but cost more to read back)
 constexpr int kYBuffers = 3;                           // rotating targets: in use, being read, being cleared
 constexpr int kSplitRotate = 41;                       // per-layer rotation of the slab split
 constexpr long long kWaitCycles = 3000000000LL;        // bound of every device-side wait (~1.5 s)
@@ -231,7 +231,8 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
     uint8_t* ring = smem;
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(ring + (size_t)p.n_slots * p.slot_bytes);
     uint64_t* empty_bar = full_bar + kMaxSlots;
-    float* red = reinterpret_cast<float*>(empty_bar + kMaxSlots);   // [NMAT][kGroupWarps][rmax]
+    uint64_t* y_bar = empty_bar + kMaxSlots;                        // completion of the read-back copy (+ 8 bytes padding)
+    float* red = reinterpret_cast<float*>(y_bar + 2);               // [NMAT][kGroupWarps][rmax]
     float* h_s = red + NMAT * kGroupWarps * p.rmax;                 // [rmax]
     float* ss_red = h_s + p.rmax;                                   // [NG][kGroupWarps]
     volatile int* abort_flag = reinterpret_cast<volatile int*>(ss_red + NG * kGroupWarps);
@@ -248,6 +249,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
             mbar_init(smem_u32(&full_bar[s]), 1);
             mbar_init(smem_u32(&empty_bar[s]), kGroupWarps);     // the warps of the group that reads the slot
         }
+        mbar_init(smem_u32(y_bar), 1);
         *abort_flag = 0;
         *layers_done = 0;
         mbar_fence_init();
@@ -525,10 +527,9 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
         }
 
         // ----------------------------------------- cross-CTA sum of partial y --
-        // Every CTA adds its partial into one of kYCopies copies of the layer's target (adds to
-        // one address are serialised in L2, so they are spread); after the grid barrier every
-        // thread sums the copies for its columns.  Targets rotate over three buffers: while layer
-        // l's is read, the one layer l+2 will use is cleared (last read before the barrier of l).
+        // Every CTA adds its partial into the layer's target; after the grid barrier every CTA
+        // reads the sum back.  Targets rotate over three buffers: while layer l's is read, the
+        // one layer l+2 will use is cleared (last read before the barrier of l).
         const bool last = (l == p.L - 1);
         float* ybase = p.ybuf + (size_t)(l % kYBuffers) * kYCopies * d;
         float* ytarget = ybase + (size_t)(cta & (kYCopies - 1)) * d;
@@ -572,6 +573,16 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
 
         grid_barrier(p.ctrl, (unsigned)(l + 1) * (unsigned)G, abort_flag, NC);
 
+        // The layer's sum comes back as one bulk copy into the buffer the partial left from (256
+        // requests of 128 bytes per CTA instead of some thousand 16-byte loads, which matters while
+        // the path to L2 is full of weight requests); every consumer waits for its completion.
+        if (tid == 0 && !*abort_flag) {
+            const uint32_t yb = smem_u32(y_bar);
+            mbar_arrive_expect_tx(yb, (uint32_t)d * (uint32_t)sizeof(float));
+            bulk_g2s(smem_u32(ysum), ybase, (uint32_t)d * (uint32_t)sizeof(float), yb);
+        }
+        wait_slot(smem_u32(y_bar), (uint32_t)(l & 1), abort_flag, p.ctrl);
+
         // ------------------------- next input: (x + y) / rms(x + y), rounded --
         float ss = 0.f;
         float2 xn[VPT][PAIRS];        // x + y in fp32, until the norm is known
@@ -582,13 +593,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
             if (v < nv) {
 #pragma unroll
                 for (int c = 0; c < PAIRS; c += 2) {
-                    float4 u[kYCopies];
-#pragma unroll
-                    for (int cp = 0; cp < kYCopies; ++cp)
-                        u[cp] = __ldcg(reinterpret_cast<const float4*>(ybase + (size_t)cp * d + (size_t)v * EPV + 2 * c));
-                    float4 t = u[0];
-#pragma unroll
-                    for (int cp = 1; cp < kYCopies; ++cp) { t.x += u[cp].x; t.y += u[cp].y; t.z += u[cp].z; t.w += u[cp].w; }
+                    const float4 t = *reinterpret_cast<const float4*>(ysum + (size_t)v * EPV + 2 * c);
                     if (cta == l % G && grp == 0) {
                         if (p.y_layers) *reinterpret_cast<float4*>(p.y_layers + (size_t)l * d + (size_t)v * EPV + 2 * c) = t;
                         if (last) *reinterpret_cast<float4*>(p.y_last + (size_t)v * EPV + 2 * c) = t;
@@ -647,7 +652,7 @@ static size_t ysum_smem_bytes(int groups, int vpt, size_t esize)
 
 static size_t fixed_smem_bytes(int rmax, bool gated, int groups)
 {
-    size_t b = 2 * kMaxSlots * sizeof(uint64_t);
+    size_t b = (2 * kMaxSlots + 2) * sizeof(uint64_t);
     b += (size_t)(gated ? 2 : 1) * kGroupWarps * rmax * sizeof(float);
     b += (size_t)rmax * sizeof(float);
     b += (size_t)groups * kGroupWarps * sizeof(float) + 16;
@@ -883,7 +888,7 @@ coreinfer_status coreinfer_ffn_decode_stack(const coreinfer_layer* layers, int32
 // scratch of the stack kernel (control words + the rotating reduction targets) lives in a
 // fixed array inside the library image.  The array costs kNoAllocScratchBytes of HBM on every
 // GPU that loads the library, for the life of the process.
-constexpr size_t kNoAllocScratchBytes = 256u << 10;   // 256 KiB: 256 + 24 * d_model bytes must fit
+constexpr size_t kNoAllocScratchBytes = 128u << 10;   // 128 KiB: 256 + 12 * d_model bytes must fit
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
 
 // The array's name is only a handle on the host; its device address comes from

@@ -44,7 +44,7 @@ def test_noalloc_matches_workspace_variant_twice_in_a_row():
 
 def test_noalloc_rejects_shapes_beyond_its_scratch():
     require_gpu()
-    cfg = wl.CONFIGS["opt6.7b"].with_(L=2, d_model=16384)        # 256 + 24 * 16384 B = 384 KiB > 256 KiB
+    cfg = wl.CONFIGS["opt6.7b"].with_(L=2, d_model=16384)        # 256 + 12 * 16384 B = 192 KiB > 128 KiB
     up, _, down = wl.compacted_weights_random(cfg, 0, 8, device="cuda")
     arr = ci.binding.make_layers([(up, None, down, None, None)] * cfg.L)
     x0 = wl.decode_input(cfg, 0, device="cuda")
