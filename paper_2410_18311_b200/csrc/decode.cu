@@ -160,8 +160,9 @@ __device__ __forceinline__ void grid_barrier(unsigned* ctrl, unsigned target, vo
 {
     named_bar_sync(1, nthreads);
     if (threadIdx.x == 0 && !*abort_flag) {
-        __threadfence();
-        atomicAdd(&ctrl[1], 1u);
+        // the arrival is a release (everything this thread has observed complete, the CTA's
+        // reduction included, is visible before it), the poll an acquire
+        red_release_add(&ctrl[1], 1u);
         const long long t0 = clock64();
         unsigned it = 0;
         for (;;) {
@@ -176,7 +177,6 @@ __device__ __forceinline__ void grid_barrier(unsigned* ctrl, unsigned target, vo
                 }
             }
         }
-        __threadfence();
     }
     named_bar_sync(1, nthreads);
 }
