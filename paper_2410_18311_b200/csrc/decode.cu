@@ -48,6 +48,7 @@ struct LayerDev {
 struct DecodeParams {
     int L, d, nv, row_bytes, slot_bytes, n_slots, rmax;
     int runahead;       // ring items of the next layer the producer may request before this layer's exchange is over
+    float inv_d;        // 1 / d_model
     int ysum_ofs;       // shared-memory offset of the buffer holding the CTA's partial y
     const void* x0;
     float* y_last;
@@ -58,11 +59,14 @@ struct DecodeParams {
     LayerDev layers[COREINFER_MAX_LAYERS];
 };
 
+// 32-bit arithmetic (a 64-bit division costs several hundred cycles per layer on the device);
+// the host refuses K * G >= 2^32.
 __host__ __device__ __forceinline__ void slab_of(int cta, int G, int layer, int K, int* k0, int* k1)
 {
-    int vc = (cta + layer * kSplitRotate) % G;
-    *k0 = (int)(((long long)vc * K) / G);
-    *k1 = (int)(((long long)(vc + 1) * K) / G);
+    const unsigned g = (unsigned)G;
+    const unsigned vc = ((unsigned)cta + (unsigned)layer * (unsigned)kSplitRotate) % g;
+    *k0 = (int)(vc * (unsigned)K / g);
+    *k1 = (int)((vc + 1u) * (unsigned)K / g);
 }
 
 // items per consumer batch for one group (register budget: 4 * items * vectors per thread)
@@ -625,7 +629,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
         float tot = 0.f;
 #pragma unroll
         for (int w = 0; w < kGroupWarps; ++w) tot += ss_red[grp * kGroupWarps + w];
-        const float inv = 1.0f / sqrtf(tot / (float)d);
+        const float inv = rsqrtf(tot * p.inv_d);     // within 2 ulp of 1 / sqrt(mean square)
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
             const int v = gt + i * kGroupThreads;
@@ -774,6 +778,9 @@ static coreinfer_status decode_stack_b1(const coreinfer_layer* layers, int L, co
         if (layers[l].K > Kmax) Kmax = layers[l].K;
     }
     p.rmax = (Kmax + G - 1) / G + 1;
+    if ((unsigned long long)Kmax * (unsigned long long)G >= (1ull << 32))
+        CI_FAIL(COREINFER_ERR_UNSUPPORTED, "K = %d is too large for the slab split (K * SM count must stay below 2^32)", Kmax);
+    p.inv_d = 1.0f / (float)d_model;
     const int groups = groups_for(p.nv);
     if ((p.nv + kGroupThreads - 1) / kGroupThreads > 8)
         CI_FAIL(COREINFER_ERR_UNSUPPORTED, "d_model %d is too wide for this kernel (max %d bytes per row)",
