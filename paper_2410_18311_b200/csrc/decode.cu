@@ -157,32 +157,27 @@ __device__ __forceinline__ bool wait_slot(uint32_t bar, uint32_t parity, volatil
     }
 }
 
-// All consumer threads call this.  The arrival counter is zeroed by the host before
-// the launch; barrier number b (0-based) completes when it reaches (b + 1) * G.
-__device__ __forceinline__ void grid_barrier(unsigned* ctrl, unsigned target, volatile int* abort_flag,
-                                             int nthreads)
+// One thread per CTA calls this.  The arrival counter is zeroed by the host before the launch;
+// barrier number b (0-based) completes when it reaches (b + 1) * G.  The arrival itself is a
+// relaxed addition: what it publishes has been ordered before it by the caller (a fence for
+// the CTA's earlier plain writes, a completion wait for its bulk reduction).
+__device__ __forceinline__ void grid_arrive_and_wait(unsigned* ctrl, unsigned target, volatile int* abort_flag)
 {
-    named_bar_sync(1, nthreads);
-    if (threadIdx.x == 0 && !*abort_flag) {
-        // the arrival is a release (everything this thread has observed complete, the CTA's
-        // reduction included, is visible before it), the poll an acquire
-        red_release_add(&ctrl[1], 1u);
-        const long long t0 = clock64();
-        unsigned it = 0;
-        for (;;) {
-            if (ld_acquire_gpu(&ctrl[1]) >= target) break;
-            __nanosleep(32);
-            if ((++it & 255u) == 0u) {             // now and then: has another CTA given up? out of time?
-                if (ld_acquire_gpu(&ctrl[0]) != kStatusOk) { *abort_flag = 1; break; }
-                if (clock64() - t0 > kWaitCycles) {
-                    *abort_flag = 1;
-                    atomicMax(&ctrl[0], (unsigned)kStatusTimeout);
-                    break;
-                }
+    red_relaxed_add(&ctrl[1], 1u);
+    const long long t0 = clock64();
+    unsigned it = 0;
+    for (;;) {
+        if (ld_acquire_gpu(&ctrl[1]) >= target) break;
+        __nanosleep(32);
+        if ((++it & 255u) == 0u) {             // now and then: has another CTA given up? out of time?
+            if (ld_acquire_gpu(&ctrl[0]) != kStatusOk) { *abort_flag = 1; break; }
+            if (clock64() - t0 > kWaitCycles) {
+                *abort_flag = 1;
+                atomicMax(&ctrl[0], (unsigned)kStatusTimeout);
+                break;
             }
         }
     }
-    named_bar_sync(1, nthreads);
 }
 
 // 8 values per lane -> 8 warp totals, one per group of 4 lanes (9 shuffles).
@@ -570,20 +565,26 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
             fence_proxy_async();          // these generic-proxy writes are read by the copy engine next
         }
         named_bar_sync(1, NC);
-        if (tid == 0 && !*abort_flag) {
-            bulk_reduce_add_f32(ytarget, smem_u32(ysum), (uint32_t)d * (uint32_t)sizeof(float));
-            bulk_wait_all();
-        }
-
-        grid_barrier(p.ctrl, (unsigned)(l + 1) * (unsigned)G, abort_flag, NC);
-
-        // The layer's sum comes back as one bulk copy into the buffer the partial left from (256
-        // requests of 128 bytes per CTA instead of some thousand 16-byte loads, which matters while
-        // the path to L2 is full of weight requests); every consumer waits for its completion.
-        if (tid == 0 && !*abort_flag) {
-            const uint32_t yb = smem_u32(y_bar);
-            mbar_arrive_expect_tx(yb, (uint32_t)d * (uint32_t)sizeof(float));
-            bulk_g2s(smem_u32(ysum), ybase, (uint32_t)d * (uint32_t)sizeof(float), yb);
+        // One thread runs the exchange: the CTA's reduction, its arrival at the grid barrier, the
+        // wait for everybody else's, and the copy that brings the sum back; the others sleep on
+        // that copy's barrier.  The fence orders the CTA's earlier plain writes to global memory
+        // (the cleared target of a later layer, made known to this thread by the CTA barriers
+        // since) before the arrival and runs while the reduction is under way; the reduction
+        // itself has been performed in L2, where every CTA reads it, once wait_group returns.
+        // The sum comes back as one bulk copy into the buffer the partial left from (256 requests
+        // of 128 bytes per CTA instead of some thousand 16-byte loads).
+        if (tid == 0) {
+            if (!*abort_flag) {
+                bulk_reduce_add_f32(ytarget, smem_u32(ysum), (uint32_t)d * (uint32_t)sizeof(float));
+                fence_acq_rel_gpu();
+                bulk_wait_all();
+                grid_arrive_and_wait(p.ctrl, (unsigned)(l + 1) * (unsigned)G, abort_flag);
+            }
+            if (!*abort_flag) {
+                const uint32_t yb = smem_u32(y_bar);
+                mbar_arrive_expect_tx(yb, (uint32_t)d * (uint32_t)sizeof(float));
+                bulk_g2s(smem_u32(ysum), ybase, (uint32_t)d * (uint32_t)sizeof(float), yb);
+            }
         }
         wait_slot(smem_u32(y_bar), (uint32_t)(l & 1), abort_flag, p.ctrl);
 
