@@ -120,13 +120,10 @@ __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p)
     return v;
 }
 
-__device__ __forceinline__ void red_relaxed_add(unsigned* p, unsigned v)
+// Arrival on a counter with release semantics at GPU scope (no value returned).
+__device__ __forceinline__ void red_release_add(unsigned* p, unsigned v)
 {
-    asm volatile("red.relaxed.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
-__device__ __forceinline__ void fence_acq_rel_gpu()
-{
-    asm volatile("fence.acq_rel.gpu;" ::: "memory");
+    asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
 __device__ __forceinline__ void red_add_v4(float* p, float a, float b, float c, float d)

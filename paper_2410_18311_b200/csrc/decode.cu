@@ -157,13 +157,14 @@ __device__ __forceinline__ bool wait_slot(uint32_t bar, uint32_t parity, volatil
     }
 }
 
-// One thread per CTA calls this.  The arrival counter is zeroed by the host before the launch;
-// barrier number b (0-based) completes when it reaches (b + 1) * G.  The arrival itself is a
-// relaxed addition: what it publishes has been ordered before it by the caller (a fence for
-// the CTA's earlier plain writes, a completion wait for its bulk reduction).
+// One thread per CTA calls this, after it has seen the CTA's work complete.  The arrival
+// counter is zeroed by the host before the launch; barrier number b (0-based) completes when it
+// reaches (b + 1) * G.  The arrival is a release at GPU scope (what this thread has observed,
+// the completed bulk reduction and the CTA's earlier plain writes included, becomes visible
+// before it), the poll an acquire.
 __device__ __forceinline__ void grid_arrive_and_wait(unsigned* ctrl, unsigned target, volatile int* abort_flag)
 {
-    red_relaxed_add(&ctrl[1], 1u);
+    red_release_add(&ctrl[1], 1u);
     const long long t0 = clock64();
     unsigned it = 0;
     for (;;) {
@@ -565,18 +566,16 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
             fence_proxy_async();          // these generic-proxy writes are read by the copy engine next
         }
         named_bar_sync(1, NC);
-        // One thread runs the exchange: the CTA's reduction, its arrival at the grid barrier, the
-        // wait for everybody else's, and the copy that brings the sum back; the others sleep on
-        // that copy's barrier.  The fence orders the CTA's earlier plain writes to global memory
-        // (the cleared target of a later layer, made known to this thread by the CTA barriers
-        // since) before the arrival and runs while the reduction is under way; the reduction
-        // itself has been performed in L2, where every CTA reads it, once wait_group returns.
-        // The sum comes back as one bulk copy into the buffer the partial left from (256 requests
-        // of 128 bytes per CTA instead of some thousand 16-byte loads).
+        // One thread runs the exchange: the CTA's reduction and the wait for its completion, the
+        // arrival at the grid barrier (a release: the CTA's earlier plain writes to global memory,
+        // such as the cleared target of a later layer, are known to this thread through the CTA
+        // barriers since), the wait for everybody else's arrival, and the copy that brings the
+        // sum back; the other consumers sleep on that copy's barrier.  The sum comes back as one
+        // bulk copy into the buffer the partial left from (256 requests of 128 bytes per CTA
+        // instead of some thousand 16-byte loads).
         if (tid == 0) {
             if (!*abort_flag) {
                 bulk_reduce_add_f32(ytarget, smem_u32(ysum), (uint32_t)d * (uint32_t)sizeof(float));
-                fence_acq_rel_gpu();
                 bulk_wait_all();
                 grid_arrive_and_wait(p.ctrl, (unsigned)(l + 1) * (unsigned)G, abort_flag);
             }
@@ -589,8 +588,9 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
         wait_slot(smem_u32(y_bar), (uint32_t)(l & 1), abort_flag, p.ctrl);
 
         // ------------------------- next input: (x + y) / rms(x + y), rounded --
-        float ss = 0.f;
+        float ssp[4] = {0.f, 0.f, 0.f, 0.f};   // four chains of the sum of squares
         float2 xn[VPT][PAIRS];        // x + y in fp32, until the norm is known
+        const bool writer = (cta == l % G) && grp == 0;   // the CTA that stores this layer's y
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
             const int v = gt + i * kGroupThreads;
@@ -599,7 +599,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
 #pragma unroll
                 for (int c = 0; c < PAIRS; c += 2) {
                     const float4 t = *reinterpret_cast<const float4*>(ysum + (size_t)v * EPV + 2 * c);
-                    if (cta == l % G && grp == 0) {
+                    if (writer) {
                         if (p.y_layers) *reinterpret_cast<float4*>(p.y_layers + (size_t)l * d + (size_t)v * EPV + 2 * c) = t;
                         if (last) *reinterpret_cast<float4*>(p.y_last + (size_t)v * EPV + 2 * c) = t;
                     }
@@ -610,11 +610,12 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
                 }
 #pragma unroll
                 for (int c = 0; c < PAIRS; ++c) {
-                    ss = fmaf(xn[i][c].x, xn[i][c].x, ss);
-                    ss = fmaf(xn[i][c].y, xn[i][c].y, ss);
+                    ssp[(2 * c) & 3] = fmaf(xn[i][c].x, xn[i][c].x, ssp[(2 * c) & 3]);
+                    ssp[(2 * c + 1) & 3] = fmaf(xn[i][c].y, xn[i][c].y, ssp[(2 * c + 1) & 3]);
                 }
             }
         }
+        float ss = (ssp[0] + ssp[1]) + (ssp[2] + ssp[3]);
         {   // clear the target that layer l + 2 will use
             float4* z = reinterpret_cast<float4*>(p.ybuf + (size_t)((l + 2) % kYBuffers) * kYCopies * d);
             const int n4 = kYCopies * d / 4;
