@@ -583,6 +583,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
                 const uint32_t yb = smem_u32(y_bar);
                 mbar_arrive_expect_tx(yb, (uint32_t)d * (uint32_t)sizeof(float));
                 bulk_g2s(smem_u32(ysum), ybase, (uint32_t)d * (uint32_t)sizeof(float), yb);
+                *layers_done = l + 1;     // the exchange's last request is on its way: the producer may go on
             }
         }
         wait_slot(smem_u32(y_bar), (uint32_t)(l & 1), abort_flag, p.ctrl);
@@ -627,7 +628,6 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
         for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
         if (lane == 0) ss_red[grp * kGroupWarps + gw] = ss;
         named_bar_sync(2 + grp, kGroupThreads);
-        if (tid == 0) *layers_done = l + 1;       // group 0 has read the sum: the producer may go on
         float tot = 0.f;
 #pragma unroll
         for (int w = 0; w < kGroupWarps; ++w) tot += ss_red[grp * kGroupWarps + w];
@@ -800,7 +800,10 @@ static coreinfer_status decode_stack_b1(const coreinfer_layer* layers, int L, co
     if (groups == 2 && slots >= 2 * batch) slots -= slots % (2 * batch);
     p.n_slots = (int)slots;
     const size_t smem = fixed + (size_t)p.n_slots * p.slot_bytes;
-    p.runahead = 16;      // measured at the OPT-6.7B shape: 16 of the 24 slots beats both 8 and no limit
+    // Measured on the four model shapes: about 100 KB of the next layer requested ahead of the
+    // exchange is best (12 rows of 8 or 10 KB; 4-5 rows of 18 KB); more delays the exchange's own
+    // messages, less leaves the ring empty when the consumers come back.
+    p.runahead = p.slot_bytes <= 12 * 1024 ? 12 : (96 * 1024 / p.slot_bytes < 4 ? 4 : 96 * 1024 / p.slot_bytes);
     p.ysum_ofs = (int)((size_t)p.n_slots * p.slot_bytes + fixed0);
     p.x0 = x0;
     p.y_last = y_last;
