@@ -581,8 +581,8 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
             }
             if (!*abort_flag) {
                 const uint32_t yb = smem_u32(y_bar);
-                mbar_arrive_expect_tx(yb, (uint32_t)d * (uint32_t)sizeof(float));
-                bulk_g2s(smem_u32(ysum), ybase, (uint32_t)d * (uint32_t)sizeof(float), yb);
+                mbar_arrive_expect_tx(yb, (uint32_t)(kYCopies * d) * (uint32_t)sizeof(float));
+                bulk_g2s(smem_u32(ysum), ybase, (uint32_t)(kYCopies * d) * (uint32_t)sizeof(float), yb);
                 *layers_done = l + 1;     // the exchange's last request is on its way: the producer may go on
             }
         }
@@ -599,7 +599,12 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
             if (v < nv) {
 #pragma unroll
                 for (int c = 0; c < PAIRS; c += 2) {
-                    const float4 t = *reinterpret_cast<const float4*>(ysum + (size_t)v * EPV + 2 * c);
+                    float4 t = *reinterpret_cast<const float4*>(ysum + (size_t)v * EPV + 2 * c);
+#pragma unroll
+                    for (int cp = 1; cp < kYCopies; ++cp) {
+                        const float4 o = *reinterpret_cast<const float4*>(ysum + (size_t)cp * d + (size_t)v * EPV + 2 * c);
+                        t.x += o.x; t.y += o.y; t.z += o.z; t.w += o.w;
+                    }
                     if (writer) {
                         if (p.y_layers) *reinterpret_cast<float4*>(p.y_layers + (size_t)l * d + (size_t)v * EPV + 2 * c) = t;
                         if (last) *reinterpret_cast<float4*>(p.y_last + (size_t)v * EPV + 2 * c) = t;
@@ -653,7 +658,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
 static size_t ysum_smem_bytes(int groups, int vpt, size_t esize)
 {
     (void)groups;
-    return (size_t)vpt * kGroupThreads * (16 / esize) * sizeof(float);
+    return (size_t)kYCopies * vpt * kGroupThreads * (16 / esize) * sizeof(float);   // room for the copies read back
 }
 
 static size_t fixed_smem_bytes(int rmax, bool gated, int groups)
