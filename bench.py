@@ -27,10 +27,10 @@ METRIC = "core-sparse decode tokens/s at batch 1; achieved HBM GB/s vs B200 peak
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode_stack_kernel launch at the bench
-# workload: measured by ncu on a 4-layer launch of the same shapes (219.45 MB) and scaled by the
+# workload: measured by ncu on a 4-layer launch of the same shapes (219.12 MB) and scaled by the
 # layer count, since every layer streams its own weights (profiles/decode_stack_kernel_opt6.7b.md).
 # Set to None whenever the kernel changes until the capture is repeated.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"opt6.7b": 219.45e6 / 4 * 32}
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"opt6.7b": 219.12e6 / 4 * 32}
 
 
 def parse_args():

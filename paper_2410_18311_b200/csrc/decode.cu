@@ -16,12 +16,14 @@
 // of at most 8 KB two such groups take alternate batches, so that one group's shared-memory
 // reads overlap the other's arithmetic; wider rows use one group.
 //
-// Exchange per layer: every group adds its partial y (d_model fp32) into a global vector with
-// vector reductions, then all CTAs meet at a grid barrier, read the full y, and every group
-// forms the next layer's input redundantly in registers.  Every wait (slot barriers, grid
-// barrier) is bounded: when one gives up, the CTA marks the workspace status word, stops
-// waiting everywhere, runs the rest of its schedule without synchronising on data, drains its
-// own copies in flight and returns.
+// Exchange per layer: the CTA's partial y (d_model fp32) is assembled in shared memory and added
+// into a global vector with one bulk reduction; one thread waits for it, arrives at a grid
+// barrier (release), polls for everybody else's arrival (acquire) and brings the sum back with
+// one bulk copy, on whose barrier the other consumers sleep; every group then forms the next
+// layer's input redundantly in registers.  Every wait (slot barriers, grid barrier, read-back)
+// is bounded: when one gives up, the CTA marks the workspace status word, stops waiting
+// everywhere, runs the rest of its schedule without synchronising on data, drains its own
+// copies in flight and returns.
 #include "common.cuh"
 
 namespace coreinfer {
