@@ -49,7 +49,6 @@ struct LayerDev {
 
 struct DecodeParams {
     int L, d, nv, row_bytes, slot_bytes, n_slots, rmax;
-    int n_slots0;       // slots of the first consumer group's ring (the second group's: the rest; one group: all)
     int runahead;       // ring items of the next layer the producer may request before this layer's exchange is over
     float inv_d;        // 1 / d_model
     int ysum_ofs;       // shared-memory offset of the buffer holding the CTA's partial y
@@ -265,15 +264,10 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
     // "empty" barrier), so the latency of one issue is not the issue rate.
     if (tid >= NC) {
         const int lane = tid - NC;
-        // Each consumer group has a ring of its own (ring g: slots base[g] .. base[g] + size[g] - 1):
-        // a slot then always serves the same group, whatever the slot count, and no group ever
-        // tests a barrier that another group's progress decides (a parity test on a barrier a
-        // full ring pass behind would report "complete").
-        const int size0 = p.n_slots0, size1 = NS - p.n_slots0;
-        const int round_max = size0 < 8 ? size0 : 8;
-        int cur0 = 0, cur1 = 0;             // ring position of the next item of each group
-        uint32_t par0 = 0, par1 = 0;        // parity of the ring pass that position belongs to
-        long long issued0 = 0, issued1 = 0;
+        const int round_max = NS < 8 ? NS : 8;
+        int slot0 = 0;                // ring position of the round's first item
+        uint32_t phase0 = 0;          // parity of the ring pass that position belongs to
+        long long issued = 0;
         for (int l = 0; l < p.L; ++l) {
             const LayerDev& ly = p.layers[l];
             int k0, k1;
@@ -281,10 +275,6 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
             const int n = k1 - k0;
             const int n_up = n * NMAT;            // items of the up (+ gate) phase
             const int total = n_up + n;           // + the down rows
-            // group of stream item q: batches of BATCH items alternate within each phase
-            auto group_of = [&](int q) -> int {
-                return NG == 1 ? 0 : (((q < n_up ? q : q - n_up) / BATCH) & 1);
-            };
             for (int q0 = 0, cnt = 0; q0 < total; q0 += cnt) {
                 if (*abort_flag) break;
                 cnt = min(round_max, total - q0);
@@ -303,16 +293,6 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
                         }
                     }
                 }
-                // items of the round per group, and those before this lane's in its group
-                int n0 = 0, n1 = 0;
-                int before = 0;
-                const int my_g = group_of(q0 + (lane < cnt ? lane : 0));
-                for (int j = 0; j < cnt; ++j) {
-                    const int g = group_of(q0 + j);
-                    n0 += (g == 0);
-                    n1 += (g == 1);
-                    if (j < lane && g == my_g) ++before;
-                }
                 if (lane < cnt) {
                     const int q = q0 + lane;
                     const uint8_t* src;
@@ -322,11 +302,9 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
                     } else {
                         src = ly.down + (size_t)(k0 + q - n_up) * p.row_bytes;
                     }
-                    const int size = my_g ? size1 : size0;
-                    int sl = (my_g ? cur1 : cur0) + before;
-                    uint32_t ph = my_g ? par1 : par0;
-                    if (sl >= size) { sl -= size; ph ^= 1u; }
-                    sl += my_g ? size0 : 0;
+                    int sl = slot0 + lane;
+                    uint32_t ph = phase0;
+                    if (sl >= NS) { sl -= NS; ph ^= 1u; }
                     if (wait_slot(smem_u32(&empty_bar[sl]), ph ^ 1u, abort_flag, p.ctrl)) {
                         const uint32_t fb = smem_u32(&full_bar[sl]);
                         mbar_arrive_expect_tx(fb, (uint32_t)p.row_bytes);
@@ -334,23 +312,16 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
                     }
                 }
                 __syncwarp();
-                cur0 += n0;
-                if (cur0 >= size0) { cur0 -= size0; par0 ^= 1u; }
-                issued0 += n0;
-                cur1 += n1;
-                if (size1 > 0 && cur1 >= size1) { cur1 -= size1; par1 ^= 1u; }
-                issued1 += n1;
+                slot0 += cnt;
+                if (slot0 >= NS) { slot0 -= NS; phase0 ^= 1u; }
+                issued += cnt;
             }
         }
         // Do not leave while a copy into this CTA's shared memory is in flight: wait (bounded)
         // for the last copy issued into every slot.  (After an abort a counted item may not have
         // been issued; its wait then runs into the bound, which only delays the return.)
         for (int sl = lane; sl < NS; sl += 32) {
-            const int g = sl >= size0 ? 1 : 0;
-            const int size = g ? size1 : size0;
-            const int local = sl - (g ? size0 : 0);
-            const long long iss = g ? issued1 : issued0;
-            const long long uses = iss / size + (local < (int)(iss % size) ? 1 : 0);
+            const long long uses = issued / NS + (sl < (int)(issued % NS) ? 1 : 0);
             if (uses == 0) continue;
             const uint32_t fb = smem_u32(&full_bar[sl]);
             const uint32_t ph = (uint32_t)((uses - 1) & 1);
@@ -383,11 +354,12 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
         if (p.x_layers && cta == 0 && grp == 0 && v < nv) reinterpret_cast<uint4*>(p.x_layers)[v] = q;
     }
 
-    // this group's ring: slots RB .. RB + RS - 1, walked in the order of the group's own items
-    const int RB = grp ? p.n_slots0 : 0;
-    const int RS = grp ? NS - p.n_slots0 : p.n_slots0;
-    int slot = 0;                 // position in the group's ring of its next item
+    int slot = 0;                 // ring position of the next item of the stream
     uint32_t phase = 0;
+    auto skip_n = [&](int n) {    // items that belong to the other group
+        slot += n;
+        if (slot >= NS) { slot -= NS; phase ^= 1u; }
+    };
     // wait for the next n items, pull them into registers (q[j][i] = vector i of item j), free them
     auto fetch = [&](uint4 (&q)[BATCH][VPT], int n) {
         {
@@ -398,15 +370,15 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
             for (int j = 0; j < BATCH; ++j) {
                 int sl = slot + (j < n ? j : 0);
                 uint32_t ph = phase;
-                if (sl >= RS) { sl -= RS; ph ^= 1u; }
-                ready &= mbar_try_wait(smem_u32(&full_bar[RB + sl]), ph);
+                if (sl >= NS) { sl -= NS; ph ^= 1u; }
+                ready &= mbar_try_wait(smem_u32(&full_bar[sl]), ph);
             }
             if (!ready) {
                 int sl = slot;
                 uint32_t ph = phase;
                 for (int j = 0; j < n; ++j) {
-                    wait_slot(smem_u32(&full_bar[RB + sl]), ph, abort_flag, p.ctrl);
-                    if (++sl == RS) { sl = 0; ph ^= 1u; }
+                    wait_slot(smem_u32(&full_bar[sl]), ph, abort_flag, p.ctrl);
+                    if (++sl == NS) { sl = 0; ph ^= 1u; }
                 }
             }
         }
@@ -414,8 +386,8 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
 #pragma unroll
             for (int j = 0; j < BATCH; ++j) {
                 int sl = slot + j;
-                if (sl >= RS) sl -= RS;
-                const uint8_t* row = ring + (size_t)(RB + sl) * p.slot_bytes;
+                if (sl >= NS) sl -= NS;
+                const uint8_t* row = ring + (size_t)sl * p.slot_bytes;
 #pragma unroll
                 for (int i = 0; i < VPT; ++i) q[j][i] = *reinterpret_cast<const uint4*>(row + vofs[i]);
             }
@@ -423,8 +395,8 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
 #pragma unroll
             for (int j = 0; j < BATCH; ++j) {
                 int sl = slot + (j < n ? j : 0);
-                if (sl >= RS) sl -= RS;
-                const uint8_t* row = ring + (size_t)(RB + sl) * p.slot_bytes;
+                if (sl >= NS) sl -= NS;
+                const uint8_t* row = ring + (size_t)sl * p.slot_bytes;
 #pragma unroll
                 for (int i = 0; i < VPT; ++i) {
                     q[j][i] = *reinterpret_cast<const uint4*>(row + vofs[i]);
@@ -435,11 +407,10 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
         __syncwarp();
         if (lane < n && !*abort_flag) {
             int sl = slot + lane;
-            if (sl >= RS) sl -= RS;
-            mbar_arrive(smem_u32(&empty_bar[RB + sl]));
+            if (sl >= NS) sl -= NS;
+            mbar_arrive(smem_u32(&empty_bar[sl]));
         }
-        slot += n;
-        if (slot >= RS) { slot -= RS; phase ^= 1u; }
+        skip_n(n);
     };
 
     for (int l = 0; l < p.L; ++l) {
@@ -459,7 +430,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
             int first_b = 0;                      // first of them
             for (int b = 0; b < nb; ++b) {
                 const int cnt = min(BATCH, n_up - b * BATCH);
-                if (NG > 1 && (b % NG) != grp) continue;      // the other group's batch, in its own ring
+                if (NG > 1 && (b % NG) != grp) { skip_n(cnt); continue; }
                 uint4 q[BATCH][VPT];
                 fetch(q, cnt);
                 if (own == 0) first_b = b;
@@ -537,7 +508,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
             const int nb = (nrows + BATCH - 1) / BATCH;
             for (int b = 0; b < nb; ++b) {
                 const int cnt = min(BATCH, nrows - b * BATCH);
-                if (NG > 1 && (b % NG) != grp) continue;      // the other group's batch, in its own ring
+                if (NG > 1 && (b % NG) != grp) { skip_n(cnt); continue; }
                 uint4 q[BATCH][VPT];
                 fetch(q, cnt);
 #pragma unroll
@@ -831,11 +802,10 @@ static coreinfer_status decode_stack_b1(const coreinfer_layer* layers, int L, co
         CI_FAIL(COREINFER_ERR_UNSUPPORTED, "K = %d, d_model = %d do not fit in shared memory", Kmax, d_model);
     long long slots = ((long long)di.smem_optin - (long long)fixed) / p.slot_bytes;
     if (slots > kMaxSlots) slots = kMaxSlots;
+    // With two groups a slot must always come back to the same group (a group never waits on the
+    // other's items, so only then can it never be a full ring pass ahead of a barrier it tests).
+    if (groups == 2 && slots >= 2 * batch) slots -= slots % (2 * batch);
     p.n_slots = (int)slots;
-    // two groups: one ring each (the first gets the odd slot); each must hold a producer round
-    p.n_slots0 = groups == 2 ? (p.n_slots + 1) / 2 : p.n_slots;
-    if (groups == 2 && p.n_slots - p.n_slots0 < 8)
-        CI_FAIL(COREINFER_ERR_UNSUPPORTED, "K = %d, d_model = %d leave too few ring slots in shared memory", Kmax, d_model);
     const size_t smem = fixed + (size_t)p.n_slots * p.slot_bytes;
     // Measured on the four model shapes: about 100 KB of the next layer requested ahead of the
     // exchange is best (12 rows of 8 or 10 KB; 4-5 rows of 18 KB); more delays the exchange's own
