@@ -27,6 +27,8 @@ class CoreSparseStack:
         self.w_gate_c = [new(K, d) if cfg.gated else None for _ in range(L)]
         self.w_downT_c = [new(K, d) for _ in range(L)]
         self.select_ws = None
+        self._side = None               # side stream and events of prefill(), created on first use
+        self._events = None
         self.stack_ws = new(B.coreinfer_ffn_decode_stack_workspace_bytes(L, 1, d, K), dtype=torch.uint8)
         self.layer_ws = new(B.coreinfer_ffn_decode_workspace_bytes(B.MAX_BATCH, d, K), dtype=torch.uint8)
         self.layers = B.make_layers([(self.w_up_c[l], self.w_gate_c[l], self.w_downT_c[l], None, None)
@@ -51,11 +53,31 @@ class CoreSparseStack:
         B.coreinfer_compact(w_up, w_gate, w_down, None, self.core_idx[l], self.K, self.w_up_c[l],
                             self.w_gate_c[l], self.w_downT_c[l], None, stream)
 
-    def prefill(self, acts, weights, stream=None):
-        """acts[l]: [T, d_ff] fp32 activations of layer l; weights[l] = (w_up, w_gate | None, w_down)."""
+    def prefill(self, acts, weights, stream=None, overlap=True):
+        """acts[l]: [T, d_ff] fp32 activations of layer l; weights[l] = (w_up, w_gate | None, w_down).
+
+        Selection is a chain of small latency-bound kernels, compaction is bandwidth-bound: with
+        `overlap` the compaction of layer l runs on a side stream while `stream` goes on with the
+        selection of layer l + 1.  On return `stream` has been made to wait for the side stream."""
+        main = torch.cuda.current_stream() if stream is None else stream
+        if not overlap:
+            for l in range(self.cfg.L):
+                self.select_layer(l, acts[l], None, main)
+                self.compact_layer(l, *weights[l], stream=main)
+            return
+        if self._side is None:
+            self._side = torch.cuda.Stream(device=self.core_idx[0].device)
+            self._events = [torch.cuda.Event() for _ in range(self.cfg.L + 2)]
+        side, ev = self._side, self._events
+        ev[-2].record(main)                 # earlier work on `stream` may still read the compacted buffers
+        side.wait_event(ev[-2])
         for l in range(self.cfg.L):
-            self.select_layer(l, acts[l], None, stream)
-            self.compact_layer(l, *weights[l], stream=stream)
+            self.select_layer(l, acts[l], None, main)
+            ev[l].record(main)
+            side.wait_event(ev[l])
+            self.compact_layer(l, *weights[l], stream=side)
+        ev[-1].record(side)
+        main.wait_event(ev[-1])
 
     def decode(self, x0, y_last, y_layers=None, x_layers=None, stream=None):
         """x0 [1, d] -> y_last [1, d] fp32 (FFN output of the last layer)."""
