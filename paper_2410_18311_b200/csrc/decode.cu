@@ -540,58 +540,32 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
         // engine adds the whole vector into the target (L2 then sees 128-byte line reductions
         // instead of a thousand 16-byte atomics per CTA, whose acknowledgements a fence had to
         // wait for).
-        auto cell_of = [&](int i, int c) -> float4* {
-            return reinterpret_cast<float4*>(ysum + (size_t)(gt + i * kGroupThreads) * EPV + 2 * c);
-        };
-        if (NG == 2 && VPT % 2 == 0) {
-            // Both groups hold a partial for every column.  Each first stores the half of its
-            // vectors that the other group will finish, then adds its own values onto what the
-            // other stored for its half: the two groups work side by side.
+        if (NG == 2) {
+            if (grp == 1) {
 #pragma unroll
-            for (int i = 0; i < VPT; ++i)
-                if ((i & 1) != grp) {
+                for (int i = 0; i < VPT; ++i)
 #pragma unroll
                     for (int c = 0; c < PAIRS; c += 2)
-                        *cell_of(i, c) = make_float4(yacc[i][c].x, yacc[i][c].y, yacc[i][c + 1].x, yacc[i][c + 1].y);
-                }
+                        *reinterpret_cast<float4*>(ysum + (size_t)(gt + i * kGroupThreads) * EPV + 2 * c) =
+                            make_float4(yacc[i][c].x, yacc[i][c].y, yacc[i][c + 1].x, yacc[i][c + 1].y);
+            }
             named_bar_sync(1, NC);
+        }
+        if (grp == 0) {
 #pragma unroll
-            for (int i = 0; i < VPT; ++i)
-                if ((i & 1) == grp) {
+            for (int i = 0; i < VPT; ++i) {
 #pragma unroll
-                    for (int c = 0; c < PAIRS; c += 2) {
-                        float4 t = *cell_of(i, c);
-                        t.x += yacc[i][c].x; t.y += yacc[i][c].y; t.z += yacc[i][c + 1].x; t.w += yacc[i][c + 1].y;
-                        *cell_of(i, c) = t;
+                for (int c = 0; c < PAIRS; c += 2) {
+                    float4* cell = reinterpret_cast<float4*>(ysum + (size_t)(gt + i * kGroupThreads) * EPV + 2 * c);
+                    float4 t = make_float4(yacc[i][c].x, yacc[i][c].y, yacc[i][c + 1].x, yacc[i][c + 1].y);
+                    if (NG == 2) {
+                        const float4 o = *cell;
+                        t.x += o.x; t.y += o.y; t.z += o.z; t.w += o.w;
                     }
+                    *cell = t;
                 }
+            }
             fence_proxy_async();          // these generic-proxy writes are read by the copy engine next
-        } else {
-            if (NG == 2) {
-                if (grp == 1) {
-#pragma unroll
-                    for (int i = 0; i < VPT; ++i)
-#pragma unroll
-                        for (int c = 0; c < PAIRS; c += 2)
-                            *cell_of(i, c) = make_float4(yacc[i][c].x, yacc[i][c].y, yacc[i][c + 1].x, yacc[i][c + 1].y);
-                }
-                named_bar_sync(1, NC);
-            }
-            if (grp == 0) {
-#pragma unroll
-                for (int i = 0; i < VPT; ++i) {
-#pragma unroll
-                    for (int c = 0; c < PAIRS; c += 2) {
-                        float4 t = make_float4(yacc[i][c].x, yacc[i][c].y, yacc[i][c + 1].x, yacc[i][c + 1].y);
-                        if (NG == 2) {
-                            const float4 o = *cell_of(i, c);
-                            t.x += o.x; t.y += o.y; t.z += o.z; t.w += o.w;
-                        }
-                        *cell_of(i, c) = t;
-                    }
-                }
-                fence_proxy_async();      // these generic-proxy writes are read by the copy engine next
-            }
         }
         named_bar_sync(1, NC);
         // One thread runs the exchange: the CTA's reduction and the wait for its completion, the
