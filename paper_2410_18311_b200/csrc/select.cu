@@ -325,13 +325,18 @@ select_count_kernel(const uint16_t* __restrict__ partial, int G, int n4, int N, 
 // found with the same histogram search as a row threshold (12 high bits of the count, then, for
 // counts of 4096 and more, the low bits); the members are then f > c* plus the lowest-index
 // f == c* until K are taken, written in ascending index with two block scans.
+// Counts crowd into a few dozen values (near alpha * beta-ish * T), so a block-wide histogram would
+// serialise thousands of shared-memory atomics on the same few words.  When the first-pass bins
+// fit, every warp counts into a histogram of its own (`wstride` > 0: words per warp) and the 32
+// of them are added up afterwards.
 __global__ void __launch_bounds__(kSelThreads, 1)
-select_top_kernel(const int32_t* __restrict__ f, int N, int K, int T, int32_t* __restrict__ S)
+select_top_kernel(const int32_t* __restrict__ f, int N, int K, int T, int32_t* __restrict__ S, int wstride)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     int* fs = reinterpret_cast<int*>(smem);                               // [N]
     int* hist = fs + ((N + 3) & ~3);                                      // [kSelBins]
     SelShared* sh = reinterpret_cast<SelShared*>(hist + kSelBins);
+    int* whist = reinterpret_cast<int*>(sh + 1);                          // [kSelWarps][wstride]
     const int tid = threadIdx.x;
     for (int i = tid; i < N; i += kSelThreads) fs[i] = f[i];
     const int C = (N + kSelThreads - 1) / kSelThreads;
@@ -341,14 +346,30 @@ select_top_kernel(const int32_t* __restrict__ f, int N, int K, int T, int32_t* _
     while ((T >> shift) >= kSelBins) ++shift;
     int cstar = 0, above = 0, need = K;
     for (int pass = 0; pass < (shift > 0 ? 2 : 1); ++pass) {
-        for (int i = tid; i < kSelBins; i += kSelThreads) hist[i] = 0;
-        __syncthreads();
-        for (int n = n0; n < n1; ++n) {
-            const int v = fs[n];
-            if (pass == 0) atomicAdd(&hist[v >> shift], 1);
-            else if ((v >> shift) == (cstar >> shift)) atomicAdd(&hist[v & ((1 << shift) - 1)], 1);
+        if (pass == 0 && wstride > 0) {
+            for (int i = tid; i < kSelWarps * wstride; i += kSelThreads) whist[i] = 0;
+            __syncthreads();
+            int* mine = whist + (tid >> 5) * wstride;
+            for (int n = n0; n < n1; ++n) atomicAdd(&mine[fs[n] >> shift], 1);
+            __syncthreads();
+            const int nb = (T >> shift) + 1;
+            for (int b = tid; b < kSelBins; b += kSelThreads) {
+                int c = 0;
+                if (b < nb)
+                    for (int w = 0; w < kSelWarps; ++w) c += whist[w * wstride + b];
+                hist[b] = c;
+            }
+            __syncthreads();
+        } else {
+            for (int i = tid; i < kSelBins; i += kSelThreads) hist[i] = 0;
+            __syncthreads();
+            for (int n = n0; n < n1; ++n) {
+                const int v = fs[n];
+                if (pass == 0) atomicAdd(&hist[v >> shift], 1);
+                else if ((v >> shift) == (cstar >> shift)) atomicAdd(&hist[v & ((1 << shift) - 1)], 1);
+            }
+            __syncthreads();
         }
-        __syncthreads();
         find_bin(hist, need, false, 0.0, sh);
         cstar |= pass == 0 ? (sh->bin << shift) : sh->bin;
         above += sh->above;
@@ -466,9 +487,16 @@ coreinfer_status coreinfer_select_core(const void* act, coreinfer_dtype act_dtyp
     select_count_kernel<<<(n4 / 4 + kCountCols - 1) / kCountCols, kCountCols * kCountSlices, 0, st>>>(partial, G, n4, d_ff, f);
     CI_CUDA(cudaGetLastError());
 
-    const size_t smem_top = (size_t)n4 * sizeof(int) + kSelBins * sizeof(int) + sizeof(SelShared) + 16;
+    size_t smem_top = (size_t)n4 * sizeof(int) + kSelBins * sizeof(int) + sizeof(SelShared) + 16;
+    int top_shift = 0;
+    while ((T >> top_shift) >= kSelBins) ++top_shift;
+    int wstride = (((T >> top_shift) + 1 + 31) & ~31) + 1;        // odd: the warps' copies of a bin fall into different banks
+    if (smem_top + (size_t)kSelWarps * wstride * sizeof(int) <= (size_t)di.smem_optin)
+        smem_top += (size_t)kSelWarps * wstride * sizeof(int);
+    else
+        wstride = 0;
     CI_CUDA(cudaFuncSetAttribute(select_top_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_top));
-    select_top_kernel<<<1, kSelThreads, smem_top, st>>>(f, d_ff, K, T, core_idx);
+    select_top_kernel<<<1, kSelThreads, smem_top, st>>>(f, d_ff, K, T, core_idx, wstride);
     CI_CUDA(cudaGetLastError());
     return COREINFER_OK;
 }
