@@ -333,12 +333,15 @@ __global__ void __launch_bounds__(kSelThreads, 1)
 select_top_kernel(const int32_t* __restrict__ f, int N, int K, int T, int32_t* __restrict__ S, int wstride)
 {
     extern __shared__ __align__(128) uint8_t smem[];
-    int* fs = reinterpret_cast<int*>(smem);                               // [N]
-    int* hist = fs + ((N + 3) & ~3);                                      // [kSelBins]
+    // counts in shared memory, one pad word per 32 so that thread t's contiguous run
+    // [t*C, (t+1)*C) and its neighbours' fall into different banks
+    int* fs = reinterpret_cast<int*>(smem);                               // [N + N/32 + 1]
+    auto at = [](int n) { return n + (n >> 5); };
+    int* hist = fs + ((N + (N >> 5) + 4) & ~3);                           // [kSelBins]
     SelShared* sh = reinterpret_cast<SelShared*>(hist + kSelBins);
     int* whist = reinterpret_cast<int*>(sh + 1);                          // [kSelWarps][wstride]
     const int tid = threadIdx.x;
-    for (int i = tid; i < N; i += kSelThreads) fs[i] = f[i];
+    for (int i = tid; i < N; i += kSelThreads) fs[at(i)] = f[i];
     const int C = (N + kSelThreads - 1) / kSelThreads;
     const int n0 = min(tid * C, N), n1 = min(n0 + C, N);
 
@@ -350,7 +353,7 @@ select_top_kernel(const int32_t* __restrict__ f, int N, int K, int T, int32_t* _
             for (int i = tid; i < kSelWarps * wstride; i += kSelThreads) whist[i] = 0;
             __syncthreads();
             int* mine = whist + (tid >> 5) * wstride;
-            for (int n = n0; n < n1; ++n) atomicAdd(&mine[fs[n] >> shift], 1);
+            for (int n = n0; n < n1; ++n) atomicAdd(&mine[fs[at(n)] >> shift], 1);
             __syncthreads();
             const int nb = (T >> shift) + 1;
             for (int b = tid; b < kSelBins; b += kSelThreads) {
@@ -364,7 +367,7 @@ select_top_kernel(const int32_t* __restrict__ f, int N, int K, int T, int32_t* _
             for (int i = tid; i < kSelBins; i += kSelThreads) hist[i] = 0;
             __syncthreads();
             for (int n = n0; n < n1; ++n) {
-                const int v = fs[n];
+                const int v = fs[at(n)];
                 if (pass == 0) atomicAdd(&hist[v >> shift], 1);
                 else if ((v >> shift) == (cstar >> shift)) atomicAdd(&hist[v & ((1 << shift) - 1)], 1);
             }
@@ -379,21 +382,21 @@ select_top_kernel(const int32_t* __restrict__ f, int N, int K, int T, int32_t* _
     // need = how many f == c* are admitted, lowest index first
 
     int ce = 0;
-    for (int n = n0; n < n1; ++n) ce += fs[n] == cstar ? 1 : 0;
+    for (int n = n0; n < n1; ++n) ce += fs[at(n)] == cstar ? 1 : 0;
     int tot;
     int rank = block_excl_scan(ce, sh, &tot);
     int cm = 0;
     {
         int r = rank;
         for (int n = n0; n < n1; ++n) {
-            const int v = fs[n];
+            const int v = fs[at(n)];
             if (v > cstar) ++cm;
             else if (v == cstar) { cm += (r < need) ? 1 : 0; ++r; }
         }
     }
     int pos = block_excl_scan(cm, sh, &tot);
     for (int n = n0; n < n1; ++n) {
-        const int v = fs[n];
+        const int v = fs[at(n)];
         bool m = v > cstar;
         if (v == cstar) { m = rank < need; ++rank; }
         if (m) S[pos++] = n;
@@ -487,7 +490,7 @@ coreinfer_status coreinfer_select_core(const void* act, coreinfer_dtype act_dtyp
     select_count_kernel<<<(n4 / 4 + kCountCols - 1) / kCountCols, kCountCols * kCountSlices, 0, st>>>(partial, G, n4, d_ff, f);
     CI_CUDA(cudaGetLastError());
 
-    size_t smem_top = (size_t)n4 * sizeof(int) + kSelBins * sizeof(int) + sizeof(SelShared) + 16;
+    size_t smem_top = ((size_t)n4 + n4 / 32 + 8) * sizeof(int) + kSelBins * sizeof(int) + sizeof(SelShared) + 16;
     int top_shift = 0;
     while ((T >> top_shift) >= kSelBins) ++top_shift;
     int wstride = (((T >> top_shift) + 1 + 31) & ~31) + 1;        // odd: the warps' copies of a bin fall into different banks
