@@ -148,3 +148,50 @@ def test_full_size_stack_in_the_bench_launch_configuration():
     assert torch.isfinite(y2).all()
     from helpers import rel_err_rms
     assert rel_err_rms(y2.cpu().numpy(), y_last.cpu().numpy()) < 0.3
+
+
+def test_prefill_side_stream_gives_the_same_sets_and_weights():
+    """prefill() may run each layer's compaction on a side stream while the next layer's selection
+    goes on: core sets and compacted weights must not depend on that, nor on being replayed from a
+    CUDA graph (the way the benchmark drives the request)."""
+    require_gpu()
+    cfg = wl.CONFIGS["tiny"].with_(L=3, T=40)
+    weights = [wl.layer_weights(cfg, l, device="cuda") for l in range(cfg.L)]
+    acts = [wl.planted_activations(cfg, l, cfg.T, device="cuda")[0] for l in range(cfg.L)]
+    stream = torch.cuda.current_stream()
+
+    def snapshot(stack):
+        torch.cuda.synchronize()
+        return [(stack.core_idx[l].cpu().numpy().copy(), raw_np(stack.w_up_c[l]).copy(), raw_np(stack.w_downT_c[l]).copy())
+                for l in range(cfg.L)]
+
+    plain = ci.pipeline.CoreSparseStack(cfg, device="cuda")
+    plain.prefill(acts, weights, stream, overlap=False)
+    ref = snapshot(plain)
+    for l in range(cfg.L):                                   # and the plain run against the oracle
+        S_o, _ = oracle.select(acts[l].cpu().numpy(), cfg.alpha, cfg.beta)
+        np.testing.assert_array_equal(ref[l][0], S_o)
+
+    over = ci.pipeline.CoreSparseStack(cfg, device="cuda")
+    over.prefill(acts, weights, stream, overlap=True)
+    got = snapshot(over)
+    for a, b in zip(ref, got):
+        for u, v in zip(a, b):
+            assert u.tobytes() == v.tobytes()
+
+    graphed = ci.pipeline.CoreSparseStack(cfg, device="cuda")
+    graphed.prefill(acts, weights, stream)                   # first use outside capture (one-time set-up calls)
+    for l in range(cfg.L):
+        graphed.core_idx[l].zero_()
+        graphed.w_up_c[l].zero_()
+    cap = torch.cuda.Stream()
+    cap.wait_stream(stream)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=cap, capture_error_mode="relaxed"):
+        graphed.prefill(acts, weights, torch.cuda.current_stream())
+    stream.wait_stream(cap)
+    g.replay()
+    got = snapshot(graphed)
+    for a, b in zip(ref, got):
+        for u, v in zip(a, b):
+            assert u.tobytes() == v.tobytes()
