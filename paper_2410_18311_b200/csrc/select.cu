@@ -285,6 +285,205 @@ select_rows_kernel(const float* __restrict__ act, int T, int N, long long ld, do
     }
 }
 
+// The same selection for CTAs that walk at most 255 rows (every T up to 65280).  Differences
+// that matter for speed:
+//  * the membership counters are bytes, four to a register, so a thread can also keep all its
+//    columns of the row in registers (36 of them at d_ff = 36864).  The row buffer is free as
+//    soon as every thread has its columns, the next row's copy runs during the whole selection
+//    of this one, and no pass re-reads shared memory;
+//  * the first radix digit is the 8 exponent bits, counted in a histogram per warp (activations
+//    crowd into a handful of exponents: in one shared histogram those additions queue on the
+//    same few words), then 12 and 11 mantissa bits in the shared histogram, where the entries
+//    that are left spread evenly.
+constexpr int kWarpHistStride = 257;     // 256 exponent bins; odd so that the warps' copies of a bin use different banks
+
+template <int VPT>
+__global__ void __launch_bounds__(kSelThreads, 1)
+select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long ld, double alpha,
+                        uint16_t* __restrict__ partial, unsigned* __restrict__ status, int row_bytes)
+{
+    extern __shared__ __align__(128) uint8_t smem[];
+    const int buf_bytes = (row_bytes + 127) & ~127;
+    int* hist = reinterpret_cast<int*>(smem + buf_bytes);                        // [kSelBins]
+    int* whist = hist + kSelBins;                                                // [kSelWarps][kWarpHistStride]
+    uint64_t* bar = reinterpret_cast<uint64_t*>(whist + ((kSelWarps * kWarpHistStride + 1) & ~1));
+    SelShared* sh = reinterpret_cast<SelShared*>(bar + 1);
+
+    const int tid = threadIdx.x;
+    const int G = gridDim.x;
+    const int nvec = row_bytes / 16;
+
+    if (tid == 0) {
+        mbar_init(smem_u32(bar), 1);
+        sh->abort_flag = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+
+    int issued = 0;                        // thread 0: copies issued
+    auto issue_row = [&](int t) {          // thread 0 only
+        const uint32_t b = smem_u32(bar);
+        mbar_arrive_expect_tx(b, (uint32_t)row_bytes);
+        const uint8_t* src = reinterpret_cast<const uint8_t*>(act + (long long)t * ld);
+        const uint32_t dst = smem_u32(smem);
+        for (uint32_t off = 0; off < (uint32_t)row_bytes; off += kCopyChunk) {
+            const uint32_t n = min(kCopyChunk, (uint32_t)row_bytes - off);
+            bulk_g2s(dst + off, src + off, n, b);
+        }
+        ++issued;
+    };
+
+    uint32_t cnt8[VPT];                    // four byte counters per vector (at most 255 rows per CTA)
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) cnt8[i] = 0u;
+
+    if (tid == 0 && (int)blockIdx.x < T) issue_row(blockIdx.x);
+
+    int iter = 0;
+    for (int t = blockIdx.x; t < T; t += G, ++iter) {
+        {   // bounded wait for this row's bytes
+            const uint32_t b = smem_u32(bar);
+            const uint32_t parity = (uint32_t)(iter & 1);
+            if (!mbar_try_wait(b, parity)) {
+                const long long t0 = clock64();
+                while (!mbar_try_wait(b, parity)) {
+                    if (clock64() - t0 > kSelWaitCycles) {
+                        sh->abort_flag = 1;
+                        atomicMax(status, (unsigned)kStatusTimeout);
+                        break;
+                    }
+                }
+            }
+        }
+        __syncthreads();
+        if (sh->abort_flag) break;   // block-uniform
+
+        // this thread's columns; 0 stands for "not positive" (or beyond d_ff)
+        const uint4* row = reinterpret_cast<const uint4*>(smem);
+        uint4 held[VPT];
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) {
+            const int v = tid + i * kSelThreads;
+            uint4 q = make_uint4(0, 0, 0, 0);
+            if (v < nvec) q = row[v];
+            if (v * 4 + 0 >= N || !is_pos_bits(q.x)) q.x = 0u;
+            if (v * 4 + 1 >= N || !is_pos_bits(q.y)) q.y = 0u;
+            if (v * 4 + 2 >= N || !is_pos_bits(q.z)) q.z = 0u;
+            if (v * 4 + 3 >= N || !is_pos_bits(q.w)) q.w = 0u;
+            held[i] = q;
+        }
+        // per-warp exponent histograms start at zero (their last use ended before the barrier above)
+        for (int i = tid; i < kSelWarps * kWarpHistStride; i += kSelThreads) whist[i] = 0;
+        __syncthreads();             // every thread holds its columns: the buffer may be refilled
+        if (tid == 0 && t + G < T) issue_row(t + G);
+
+        // ---- radix select of the k-th largest positive pattern: 8 + 12 + 11 bits ----
+        uint32_t vstar = 0u;
+        int need = 0, eq_total = 0;
+        {   // exponent digit
+            int* mine = whist + (tid >> 5) * kWarpHistStride;
+#pragma unroll
+            for (int i = 0; i < VPT; ++i) {
+                const uint32_t bb[4] = {held[i].x, held[i].y, held[i].z, held[i].w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (bb[e] != 0u) atomicAdd(&mine[bb[e] >> 23], 1);
+            }
+            __syncthreads();
+            for (int b = tid; b < kSelBins; b += kSelThreads) {
+                int c = 0;
+                if (b < 256) {
+#pragma unroll 8
+                    for (int w = 0; w < kSelWarps; ++w) c += whist[w * kWarpHistStride + b];
+                }
+                hist[b] = c;
+            }
+            __syncthreads();
+            need = find_bin(hist, 0, true, alpha, sh);
+            if (need > 0) {
+                vstar = (uint32_t)sh->bin << 23;
+                need -= sh->above;
+                eq_total = sh->bin_count;
+            }
+            __syncthreads();
+        }
+#pragma unroll 1
+        for (int pass = 1; pass < 3 && need > 0; ++pass) {
+            const int shift = pass == 1 ? 11 : 0;
+            const uint32_t dmask = pass == 1 ? 0xFFFu : 0x7FFu;
+            const int pshift = pass == 1 ? 23 : 11;                   // prefix = bits >> pshift
+            for (int i = tid; i < kSelBins; i += kSelThreads) hist[i] = 0;
+            __syncthreads();
+#pragma unroll
+            for (int i = 0; i < VPT; ++i) {
+                const uint32_t bb[4] = {held[i].x, held[i].y, held[i].z, held[i].w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (bb[e] != 0u && (bb[e] >> pshift) == (vstar >> pshift))
+                        atomicAdd(&hist[(bb[e] >> shift) & dmask], 1);
+            }
+            __syncthreads();
+            need = find_bin(hist, need, false, alpha, sh);
+            vstar |= (uint32_t)sh->bin << shift;
+            need -= sh->above;
+            eq_total = sh->bin_count;
+            __syncthreads();
+        }
+
+        // ---- membership (Eq. 1) and its count (Eq. 3) ----
+        if (need == 0) {
+            // no positive entry in this row: nothing to count
+        } else if (need == eq_total) {
+#pragma unroll
+            for (int i = 0; i < VPT; ++i)     // vstar > 0, masked entries are 0
+                cnt8[i] += (held[i].x >= vstar ? 1u : 0u) | (held[i].y >= vstar ? 0x100u : 0u) |
+                           (held[i].z >= vstar ? 0x10000u : 0u) | (held[i].w >= vstar ? 0x1000000u : 0u);
+        } else {
+            // more entries equal the threshold than places left: lower index first.
+            // Index order = vector round i, then thread, then element.
+            int taken = 0;
+#pragma unroll
+            for (int i = 0; i < VPT; ++i) {
+                const uint32_t bb[4] = {held[i].x, held[i].y, held[i].z, held[i].w};
+                int c = 0;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) c += (bb[e] == vstar) ? 1 : 0;
+                int tot;
+                int rank = taken + block_excl_scan(c, sh, &tot);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    if (bb[e] > vstar) cnt8[i] += 1u << (8 * e);
+                    else if (bb[e] == vstar) { cnt8[i] += (rank < need ? 1u : 0u) << (8 * e); ++rank; }
+                }
+                taken += tot;
+            }
+        }
+        __syncthreads();   // the shared scratch is free again
+    }
+
+    // Never leave with a copy into this CTA's shared memory in flight.  On the normal path
+    // every issued copy has been waited for; after an abort this is a last bounded wait.
+    __syncthreads();
+    if (tid == 0 && issued > 0) {
+        const uint32_t ph = (uint32_t)((issued - 1) & 1);
+        const long long t0 = clock64();
+        while (!mbar_try_wait(smem_u32(bar), ph))
+            if (clock64() - t0 > kSelWaitCycles) { atomicMax(status, (unsigned)kStatusTimeout); break; }
+    }
+
+    uint16_t* out = partial + (size_t)blockIdx.x * ((size_t)nvec * 4);
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+        const int v = tid + i * kSelThreads;
+        if (v < nvec) {
+            uint2 w;
+            w.x = (cnt8[i] & 0xffu) | ((cnt8[i] & 0xff00u) << 8);
+            w.y = ((cnt8[i] >> 16) & 0xffu) | ((cnt8[i] >> 24) << 16);
+            reinterpret_cast<uint2*>(out)[v] = w;
+        }
+    }
+}
+
 // f[n] = sum over the CTAs' u16 rows.  A block covers 32 groups of 4 neurons; its 8 warps take
 // every 8th row each (so the loads of a column group are spread over 8 threads) and meet in
 // shared memory.
@@ -417,6 +616,24 @@ static coreinfer_status launch_rows(int grid, size_t smem, cudaStream_t st, cons
     return COREINFER_OK;
 }
 
+static size_t sel_fast_fixed_smem()
+{
+    return kSelBins * sizeof(int) + ((kSelWarps * kWarpHistStride + 1) & ~1) * sizeof(int) + sizeof(uint64_t) +
+           sizeof(SelShared) + 128;
+}
+
+template <int VPT>
+static coreinfer_status launch_rows_fast(int grid, size_t smem, cudaStream_t st, const float* act, int T, int N,
+                                         long long ld, double alpha, uint16_t* partial, unsigned* status,
+                                         int row_bytes)
+{
+    auto kern = select_rows_fast_kernel<VPT>;
+    CI_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    kern<<<grid, kSelThreads, smem, st>>>(act, T, N, ld, alpha, partial, status, row_bytes);
+    CI_CUDA(cudaGetLastError());
+    return COREINFER_OK;
+}
+
 }  // namespace coreinfer
 
 using namespace coreinfer;
@@ -459,6 +676,12 @@ coreinfer_status coreinfer_select_core(const void* act, coreinfer_dtype act_dtyp
     const int row_bytes = n4 * 4;
     int G = T < di.sm_count ? T : di.sm_count;
     if (G > kSelMaxCtas) G = kSelMaxCtas;
+    const size_t buf = ((size_t)row_bytes + 127) & ~(size_t)127;
+    // byte counters (the fast kernel) hold 255 rows per CTA: more CTAs than SMs where that needs it
+    int G_fast = G;
+    if ((T + G_fast - 1) / G_fast > 255) G_fast = (T + 254) / 255;
+    const bool fast = G_fast <= kSelMaxCtas && sel_fast_fixed_smem() + buf <= (size_t)di.smem_optin;
+    if (fast) G = G_fast;
     if ((T + G - 1) / G > 65535)
         CI_FAIL(COREINFER_ERR_UNSUPPORTED, "T = %d: more than 65535 rows per CTA", T);
     const int K = coreinfer_count(beta, d_ff);
@@ -468,17 +691,19 @@ coreinfer_status coreinfer_select_core(const void* act, coreinfer_dtype act_dtyp
     int32_t* f = counts_out ? counts_out : (int32_t*)(partial + (size_t)(T < kSelMaxCtas ? T : kSelMaxCtas) * n4);
     CI_CUDA(cudaMemsetAsync(workspace, 0, kSelCtrlBytes, st));
 
-    const size_t buf = ((size_t)row_bytes + 127) & ~(size_t)127;
     const size_t fixed = sel_fixed_smem();
     if (fixed + buf > (size_t)di.smem_optin)
         CI_FAIL(COREINFER_ERR_UNSUPPORTED, "a row of d_ff = %d does not fit in shared memory", d_ff);
     const int nbuf = (fixed + 2 * buf <= (size_t)di.smem_optin) ? 2 : 1;
     const size_t smem = fixed + nbuf * buf;
+    const size_t smem_fast = sel_fast_fixed_smem() + buf;
     const int vpt = (n4 / 4 + kSelThreads - 1) / kSelThreads;
 #define CI_ROWS(V)                                                                                        \
     case V:                                                                                               \
-        s = launch_rows<V>(G, smem, st, (const float*)act, T, d_ff, (long long)ld_act, alpha, partial,    \
-                           status, nbuf, row_bytes);                                                      \
+        s = fast ? launch_rows_fast<V>(G, smem_fast, st, (const float*)act, T, d_ff, (long long)ld_act,   \
+                                       alpha, partial, status, row_bytes)                                 \
+                 : launch_rows<V>(G, smem, st, (const float*)act, T, d_ff, (long long)ld_act, alpha,      \
+                                  partial, status, nbuf, row_bytes);                                      \
         break;
     switch (vpt) {
         CI_ROWS(1) CI_ROWS(2) CI_ROWS(3) CI_ROWS(4) CI_ROWS(5) CI_ROWS(6) CI_ROWS(7) CI_ROWS(8) CI_ROWS(9)
