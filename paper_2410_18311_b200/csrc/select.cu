@@ -2,15 +2,16 @@
 // Definition 2 / Eq. 2).  Three kernels, all integer work on float bit patterns, so the
 // result is exact and independent of scheduling:
 //
-//   select_rows_kernel   persistent CTAs, each walks rows t = cta, cta + G, ...  A row is
-//                        brought into shared memory by bulk copies (the next row is
-//                        prefetched when two rows fit).  Per row: count the positives P,
-//                        k = ceil(alpha P), then an MSB-first radix select (12 + 12 + 7 bits)
-//                        finds the exact bit pattern of the k-th largest positive value and
-//                        how many entries equal to it are admitted (lowest index first).
-//                        Each thread owns fixed columns of every row, so the per-neuron
-//                        membership counters of Eq. 3 live in its registers: no atomics.
-//                        At the end each CTA writes its counters as one u16 row.
+//   select_rows_*_kernel CTAs walk rows t = cta, cta + G, ...  A row is brought into shared
+//                        memory by bulk copies.  Per row: count the positives P, k = ceil(alpha P),
+//                        then an MSB-first radix select finds the exact bit pattern of the k-th
+//                        largest positive value and how many entries equal to it are admitted
+//                        (lowest index first).  Each thread owns fixed columns of every row, so
+//                        the per-neuron membership counters of Eq. 3 live in its registers: no
+//                        atomics.  At the end each CTA writes its counters as one u16 row.
+//                        Two builds: the fast one (up to 255 rows per CTA: byte counters, the
+//                        row kept in registers, digits of 8 + 12 + 11 bits) and the general one
+//                        (16-bit counters, digits of 12 + 12 + 7 bits).
 //   select_count_kernel  f[n] = sum over CTAs of those rows (int32).
 //   select_top_kernel    one CTA: the K-th largest count c* by a histogram search on the count
 //                        value, then an index-ordered scan admits f > c*, and the lowest-index

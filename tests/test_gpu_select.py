@@ -103,6 +103,18 @@ def test_many_rows_per_cta_and_alpha_beta_extremes():
     _check(A[:50], 0.0001, 1.0)                                  # k_t = 1
 
 
+@pytest.mark.parametrize("T", [40000, 66000])
+def test_more_rows_than_one_cta_counts_in_bytes(T):
+    """The row kernel counts memberships in bytes (at most 255 rows per CTA): T = 40000 needs more
+    CTAs than there are SMs for that, T = 66000 is beyond it and takes the kernel with wide
+    counters; both also exercise the two-pass search of the top-K kernel (counts above 4095)."""
+    require_gpu()
+    rng = np.random.default_rng(T)
+    A = rng.standard_normal((T, 64)).astype(np.float32)
+    A[:, :7] = np.abs(A[:, :7]) + 3.0                            # a stable subset, so counts reach T
+    _check(A, 0.4, 0.2)
+
+
 def test_device_count_rule_for_every_P():
     """Row t has exactly t positives, all distinct: membership count of row t is ceil(alpha t),
     so f summed over neurons must equal the host rule for every P in 0..N."""
