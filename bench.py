@@ -354,10 +354,21 @@ def run_ours(args, cfg):
         y_d = torch.empty((1, cfg.d_model), device=dev)
         acts_d = [torch.empty_like(a) for a in acts]
 
+        copy_stream = torch.cuda.Stream(device=dev)
+        copied = [torch.cuda.Event() for _ in range(cfg.L)]
+
         def request_e2e():
+            # activations arrive layer by layer on a copy stream; each layer is selected and
+            # compacted as soon as its activations are on the device
+            copy_stream.wait_stream(stream)
+            with torch.cuda.stream(copy_stream):
+                for l in range(cfg.L):
+                    acts_d[l].copy_(acts_h[l], non_blocking=True)
+                    copied[l].record(copy_stream)
             for l in range(cfg.L):
-                acts_d[l].copy_(acts_h[l], non_blocking=True)
-            stack.prefill(acts_d, weights, stream)
+                stream.wait_event(copied[l])
+                stack.select_layer(l, acts_d[l], None, stream)
+                stack.compact_layer(l, *weights[l], stream=stream)
             for s in range(steps_tok):
                 x_d.copy_(xs_h[s:s + 1], non_blocking=True)
                 stack.decode(x_d, y_d, stream=stream)
