@@ -157,7 +157,9 @@ coreinfer_status coreinfer_ffn_decode(const void* x, int32_t batch, coreinfer_dt
  *   x_layers   device out [L, batch, d_model] in `dtype`: every layer's input as
  *              consumed, or NULL.
  *   workspace  at least coreinfer_ffn_decode_stack_workspace_bytes().
- * batch must be 1.  1 <= L <= COREINFER_MAX_LAYERS.
+ * 1 <= batch <= COREINFER_MAX_BATCH, 1 <= L <= COREINFER_MAX_LAYERS.  batch 1 is the single
+ * persistent launch described here; 2..8 sequences (sharing the core sets) run as one batched
+ * FFN launch plus one glue launch per layer, every weight byte read once for all sequences.
  * Thread blocks of this launch wait on one another at layer boundaries; every
  * such wait is bounded, and a wait that gives up makes all blocks return early
  * and records COREINFER_ERR_TIMEOUT in the workspace (read it with

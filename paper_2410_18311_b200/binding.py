@@ -184,7 +184,7 @@ def make_layers(layers):
 
 
 def coreinfer_ffn_decode_stack(layers, x0, kind, y_last, y_layers, x_layers, workspace, stream=None):
-    """layers: a coreinfer_layer array from make_layers(); x0 [1, d_model]."""
+    """layers: a coreinfer_layer array from make_layers(); x0 [batch, d_model], batch 1..8."""
     batch, d_model = x0.shape
     _check(load().coreinfer_ffn_decode_stack(layers, len(layers), _p(x0), batch, dtype_code(x0), int(kind),
                                              d_model, _p(y_last), _p(y_layers), _p(x_layers), _p(workspace),

@@ -831,7 +831,12 @@ static coreinfer_status decode_stack_b1(const coreinfer_layer* layers, int L, co
 // decode_batch.cu
 coreinfer_status decode_batched(const void* x, int batch, coreinfer_dtype dtype, coreinfer_ffn_kind kind,
                                 int d_model, const coreinfer_layer& ly, float* y, void* workspace,
-                                cudaStream_t st);
+                                cudaStream_t st, bool clear_status);
+size_t decode_stack_batched_workspace_bytes(int batch, int d_model, int K_max);
+coreinfer_status decode_stack_batched(const coreinfer_layer* layers, int L, const void* x0, int batch,
+                                      coreinfer_dtype dtype, coreinfer_ffn_kind kind, int d_model, float* y_last,
+                                      float* y_layers, void* x_layers, void* workspace, size_t workspace_bytes,
+                                      cudaStream_t st);
 
 }  // namespace coreinfer
 
@@ -848,9 +853,10 @@ size_t coreinfer_ffn_decode_workspace_bytes(int32_t batch, int32_t d_model, int3
 
 size_t coreinfer_ffn_decode_stack_workspace_bytes(int32_t L, int32_t batch, int32_t d_model, int32_t K_max)
 {
-    (void)K_max;
     if (L < 1 || batch < 1 || d_model < 1) return 0;
-    return (size_t)batch * b1_workspace_bytes(d_model);
+    if (batch == 1) return b1_workspace_bytes(d_model);
+    if (K_max < 1) return 0;
+    return decode_stack_batched_workspace_bytes(batch, d_model, K_max);
 }
 
 coreinfer_status coreinfer_ffn_decode(const void* x, int32_t batch, coreinfer_dtype dtype,
@@ -873,7 +879,7 @@ coreinfer_status coreinfer_ffn_decode(const void* x, int32_t batch, coreinfer_dt
     if (!workspace || !aligned16(workspace)) CI_FAIL(COREINFER_ERR_WORKSPACE, "workspace is NULL or misaligned");
     if (workspace_bytes < need)
         CI_FAIL(COREINFER_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, need);
-    return decode_batched(x, batch, dtype, kind, d_model, ly, y, workspace, st);
+    return decode_batched(x, batch, dtype, kind, d_model, ly, y, workspace, st, true);
 }
 
 coreinfer_status coreinfer_ffn_decode_stack(const coreinfer_layer* layers, int32_t L, const void* x0,
@@ -884,13 +890,21 @@ coreinfer_status coreinfer_ffn_decode_stack(const coreinfer_layer* layers, int32
 {
     coreinfer_status s = check_common(x0, batch, dtype, kind, d_model);
     if (s != COREINFER_OK) return s;
-    if (batch != 1) CI_FAIL(COREINFER_ERR_UNSUPPORTED, "the stack entry point is built for batch 1 (got %d)", batch);
     if (!layers) CI_FAIL(COREINFER_ERR_INVALID_ARG, "layers is NULL");
     if (L < 1 || L > COREINFER_MAX_LAYERS)
         CI_FAIL(COREINFER_ERR_INVALID_ARG, "L = %d outside 1..%d", L, COREINFER_MAX_LAYERS);
     if (!y_last || !aligned16(y_last)) CI_FAIL(COREINFER_ERR_INVALID_ARG, "y_last is NULL or not 16-byte aligned");
     if ((y_layers && !aligned16(y_layers)) || (x_layers && !aligned16(x_layers)))
         CI_FAIL(COREINFER_ERR_INVALID_ARG, "y_layers / x_layers not 16-byte aligned");
+    if (batch > 1) {
+        // 2..8 sequences sharing the core sets: one batched FFN launch and one glue launch per layer
+        for (int l = 0; l < L; ++l) {
+            s = check_layer(layers[l], l, kind);
+            if (s != COREINFER_OK) return s;
+        }
+        return decode_stack_batched(layers, L, x0, batch, dtype, kind, d_model, y_last, y_layers, x_layers, workspace,
+                                    workspace_bytes, (cudaStream_t)cuda_stream);
+    }
     const size_t need = coreinfer_ffn_decode_stack_workspace_bytes(L, batch, d_model, 0);
     return decode_stack_b1(layers, L, x0, dtype, kind, d_model, y_last, y_layers, x_layers, workspace,
                            workspace_bytes, need, (cudaStream_t)cuda_stream);
@@ -937,13 +951,13 @@ coreinfer_status coreinfer_ffn_decode_stack_noalloc(const coreinfer_layer* layer
 {
     coreinfer_status s = check_common(x0, batch, dtype, kind, d_model);
     if (s != COREINFER_OK) return s;
-    if (batch != 1) CI_FAIL(COREINFER_ERR_UNSUPPORTED, "the stack entry point is built for batch 1 (got %d)", batch);
     if (!layers) CI_FAIL(COREINFER_ERR_INVALID_ARG, "layers is NULL");
     if (L < 1 || L > COREINFER_MAX_LAYERS)
         CI_FAIL(COREINFER_ERR_INVALID_ARG, "L = %d outside 1..%d", L, COREINFER_MAX_LAYERS);
     if (!y_last || !aligned16(y_last)) CI_FAIL(COREINFER_ERR_INVALID_ARG, "y_last is NULL or not 16-byte aligned");
     if ((y_layers && !aligned16(y_layers)) || (x_layers && !aligned16(x_layers)))
         CI_FAIL(COREINFER_ERR_INVALID_ARG, "y_layers / x_layers not 16-byte aligned");
+    if (batch != 1) CI_FAIL(COREINFER_ERR_UNSUPPORTED, "this entry point is built for batch 1 (got %d)", batch);
     const size_t need = coreinfer_ffn_decode_stack_workspace_bytes(L, batch, d_model, 0);
     if (need > kNoAllocScratchBytes)
         CI_FAIL(COREINFER_ERR_UNSUPPORTED,

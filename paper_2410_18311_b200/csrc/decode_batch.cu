@@ -181,13 +181,13 @@ coreinfer_status decode_batched_mma(const void* x, int batch, bool gated, int d_
 
 coreinfer_status decode_batched(const void* x, int batch, coreinfer_dtype dtype, coreinfer_ffn_kind kind,
                                 int d_model, const coreinfer_layer& ly, float* y, void* workspace,
-                                cudaStream_t st)
+                                cudaStream_t st, bool clear_status)
 {
     DeviceInfo di;
     coreinfer_status s = device_info(&di);
     if (s != COREINFER_OK) return s;
     const bool gated = kind == COREINFER_FFN_RELU_GATED;
-    CI_CUDA(cudaMemsetAsync(workspace, 0, kCtrlBytesB, st));   // status word
+    if (clear_status) CI_CUDA(cudaMemsetAsync(workspace, 0, kCtrlBytesB, st));   // status word
     if (dtype == COREINFER_BF16) {
         s = decode_batched_mma(x, batch, gated, d_model, ly, y, (unsigned*)workspace, di, st);
         if (s != COREINFER_ERR_UNSUPPORTED) return s;          // otherwise: shape not built there, use the plain kernels
@@ -195,6 +195,98 @@ coreinfer_status decode_batched(const void* x, int batch, coreinfer_dtype dtype,
     float* h = (float*)((uint8_t*)workspace + kCtrlBytesB);
     if (dtype == COREINFER_BF16) return run_t<__nv_bfloat16>(batch, x, gated, d_model, ly, y, h, st);
     return run_t<float>(batch, x, gated, d_model, ly, y, h, st);
+}
+
+// ------------------------------------------------------------- stack, batch 2..8 --
+static __device__ __forceinline__ float to_f(float v) { return v; }
+static __device__ __forceinline__ float to_f(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> static __device__ __forceinline__ T from_f(float v);
+template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// Glue between two layers, one CTA per sequence: x_next = round((x + y) / rms(x + y)), the same
+// formula (rsqrtf of the mean square) as in the batch-1 stack kernel.
+template <typename T>
+__global__ void __launch_bounds__(256)
+batch_glue_kernel(const T* __restrict__ x, const float* __restrict__ y, T* __restrict__ x_next,
+                  T* __restrict__ x_dump, int d, float inv_d)
+{
+    __shared__ float part[8];
+    const size_t base = (size_t)blockIdx.x * d;
+    float ss = 0.f;
+    for (int j = threadIdx.x; j < d; j += 256) {
+        const float v = to_f(x[base + j]) + y[base + j];
+        ss = fmaf(v, v, ss);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += part[w];
+    const float inv = rsqrtf(tot * inv_d);
+    for (int j = threadIdx.x; j < d; j += 256) {
+        const float v = (to_f(x[base + j]) + y[base + j]) * inv;
+        const T r = from_f<T>(v);
+        x_next[base + j] = r;
+        if (x_dump) x_dump[base + j] = r;
+    }
+}
+
+static size_t align256(size_t b) { return (b + 255) & ~(size_t)255; }
+
+// layer scratch (status word + h) | y of the current layer | two x buffers (ping-pong)
+size_t decode_stack_batched_workspace_bytes(int batch, int d_model, int K_max)
+{
+    return align256(kCtrlBytesB + (size_t)batch * K_max * sizeof(float)) + align256((size_t)batch * d_model * sizeof(float)) +
+           2 * align256((size_t)batch * d_model * sizeof(float));
+}
+
+// The stack for 2..8 sequences: per layer one batched FFN (every weight byte read once for all
+// sequences) and one glue launch.  Outputs as in the batch-1 stack: y_layers / x_layers
+// [L][batch][d_model] when given.
+coreinfer_status decode_stack_batched(const coreinfer_layer* layers, int L, const void* x0, int batch,
+                                      coreinfer_dtype dtype, coreinfer_ffn_kind kind, int d_model, float* y_last,
+                                      float* y_layers, void* x_layers, void* workspace, size_t workspace_bytes,
+                                      cudaStream_t st)
+{
+    int Kmax = 0;
+    for (int l = 0; l < L; ++l) Kmax = layers[l].K > Kmax ? layers[l].K : Kmax;
+    const size_t need = decode_stack_batched_workspace_bytes(batch, d_model, Kmax);
+    if (!workspace || !aligned16(workspace)) CI_FAIL(COREINFER_ERR_WORKSPACE, "workspace is NULL or misaligned");
+    if (workspace_bytes < need)
+        CI_FAIL(COREINFER_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, need);
+    const size_t esize = dtype_size(dtype);
+    const size_t row = (size_t)batch * d_model;
+    uint8_t* w = (uint8_t*)workspace;
+    float* ybuf = (float*)(w + align256(kCtrlBytesB + (size_t)batch * Kmax * sizeof(float)));
+    uint8_t* xbuf0 = (uint8_t*)ybuf + align256(row * sizeof(float));
+    uint8_t* xbuf1 = xbuf0 + align256(row * sizeof(float));
+    CI_CUDA(cudaMemsetAsync(workspace, 0, kCtrlBytesB, st));      // status word: sticky over the layers
+    if (x_layers) CI_CUDA(cudaMemcpyAsync(x_layers, x0, row * esize, cudaMemcpyDeviceToDevice, st));
+    const void* x_in = x0;
+    for (int l = 0; l < L; ++l) {
+        const bool last = (l == L - 1);
+        float* y_out = y_layers ? y_layers + (size_t)l * row : (last ? y_last : ybuf);
+        coreinfer_status s = decode_batched(x_in, batch, dtype, kind, d_model, layers[l], y_out, workspace, st, false);
+        if (s != COREINFER_OK) return s;
+        if (last) {
+            if (y_out != y_last) CI_CUDA(cudaMemcpyAsync(y_last, y_out, row * sizeof(float), cudaMemcpyDeviceToDevice, st));
+            break;
+        }
+        void* x_next = (l & 1) ? (void*)xbuf1 : (void*)xbuf0;
+        void* dump = x_layers ? (void*)((uint8_t*)x_layers + (size_t)(l + 1) * row * esize) : nullptr;
+        if (dtype == COREINFER_BF16)
+            batch_glue_kernel<__nv_bfloat16><<<batch, 256, 0, st>>>((const __nv_bfloat16*)x_in, y_out, (__nv_bfloat16*)x_next,
+                                                                   (__nv_bfloat16*)dump, d_model, 1.0f / (float)d_model);
+        else
+            batch_glue_kernel<float><<<batch, 256, 0, st>>>((const float*)x_in, y_out, (float*)x_next, (float*)dump,
+                                                           d_model, 1.0f / (float)d_model);
+        CI_CUDA(cudaGetLastError());
+        x_in = x_next;
+    }
+    return COREINFER_OK;
 }
 
 }  // namespace coreinfer

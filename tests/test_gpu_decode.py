@@ -121,6 +121,47 @@ def test_stack_layers_teacher_forced():
                     np.testing.assert_allclose(xl[l + 1][0], x_next, rtol=tol, atol=tol)
 
 
+@pytest.mark.parametrize("B", [2, 5, 8])
+def test_stack_of_small_batches_teacher_forced(B):
+    """The stack for 2..8 sequences that share the core sets (one batched FFN and one glue launch
+    per layer): every layer's output for every sequence against the oracle on the input that layer
+    consumed, and the glue per sequence against the oracle's.  Covers the tensor-core kernel
+    (bf16, d_model a multiple of 256) and the plain batched kernels (fp32; bf16 d_model 384)."""
+    require_gpu()
+    for dtype, gated, d, K, L in [(torch.bfloat16, True, 512, 300, 3), (torch.bfloat16, False, 1024, 257, 4),
+                                  (torch.float32, False, 768, 200, 3), (torch.bfloat16, False, 384, 100, 2)]:
+        layers_cpu = [_rand_layer(d, K + 3 * l, gated, dtype, 300 + l, bias=not gated) for l in range(L)]
+        layers_gpu = [tuple(None if t is None else t.cuda() for t in ly) for ly in layers_cpu]
+        x0 = torch.randn(B, d, generator=torch.Generator().manual_seed(19)).to(dtype)
+        kind = ci.FFN_RELU_GATED if gated else ci.FFN_RELU
+        arr = ci.binding.make_layers(layers_gpu)
+        ws = torch.empty(ci.coreinfer_ffn_decode_stack_workspace_bytes(L, B, d, K + 3 * L), dtype=torch.uint8,
+                         device="cuda")
+        y_last = torch.full((B, d), float("nan"), device="cuda")
+        y_layers = torch.full((L, B, d), float("nan"), device="cuda")
+        x_layers = torch.zeros((L, B, d), dtype=dtype, device="cuda")
+        ci.coreinfer_ffn_decode_stack(arr, x0.cuda(), kind, y_last, y_layers, x_layers, ws)
+        ci.coreinfer_workspace_status(ws)
+        yl, xl = y_layers.cpu().numpy(), to_f32_np(x_layers)
+        np.testing.assert_array_equal(xl[0], to_f32_np(x0))
+        np.testing.assert_array_equal(y_last.cpu().numpy(), yl[L - 1])
+        for l in range(L):
+            up, gate, down, bup, bdown = (to_f32_np(t) for t in layers_cpu[l])
+            y_o = oracle.ffn(xl[l], kind, up, gate, down, bup, bdown)
+            assert_ffn_close(yl[l], y_o, dtype)
+            if l + 1 < L:
+                tol = 1e-5 if dtype == torch.float32 else 2 ** -7
+                for b in range(B):
+                    x_next = torch.from_numpy(oracle.glue(xl[l][b], yl[l][b])).to(dtype).float().numpy()
+                    np.testing.assert_allclose(xl[l + 1][b], x_next, rtol=tol, atol=tol)
+        # without the per-layer dumps the result is the same up to the order of the sums
+        y2 = torch.empty((B, d), device="cuda")
+        ci.coreinfer_ffn_decode_stack(arr, x0.cuda(), kind, y2, None, None, ws)
+        ci.coreinfer_workspace_status(ws)
+        from helpers import rel_err_rms
+        assert rel_err_rms(y2.cpu().numpy(), y_last.cpu().numpy()) < 0.05      # rounding flips of x may amplify over layers
+
+
 def test_stack_matches_layer_by_layer_calls():
     require_gpu()
     cfg = wl.CONFIGS["opt6.7b"].with_(L=3)
