@@ -55,7 +55,7 @@ def test_argument_errors_are_reported_without_a_device(lib):
     assert lib.coreinfer_ffn_decode(p, 1, ci.BF16, ci.FFN_RELU_GATED, 64, 4, p, null, p, null, null, p, p, 1024, null) == ci.ERR_INVALID_ARG
     # stack: batch 2 is not built, L out of range
     layers = ci.binding.Layer * 1
-    assert lib.coreinfer_ffn_decode_stack(layers(), 1, p, 2, ci.BF16, ci.FFN_RELU, 64, p, null, null, p, 1024, null) == ci.ERR_UNSUPPORTED
+    assert lib.coreinfer_ffn_decode_stack(layers(), 1, p, 9, ci.BF16, ci.FFN_RELU, 64, p, null, null, p, 1024, null) == ci.ERR_UNSUPPORTED
     assert lib.coreinfer_ffn_decode_stack(layers(), 0, p, 1, ci.BF16, ci.FFN_RELU, 64, p, null, null, p, 1024, null) == ci.ERR_INVALID_ARG
     # dense: y without h
     assert lib.coreinfer_ffn_dense_ref(p, 4, ci.F32, ci.FFN_RELU, 8, 16, p, null, p, null, null, null, p, null) == ci.ERR_INVALID_ARG
@@ -67,3 +67,4 @@ def test_workspace_sizes(lib):
     assert ci.coreinfer_ffn_decode_workspace_bytes(1, 4096, 3277) >= 4
     assert ci.coreinfer_ffn_decode_workspace_bytes(8, 4096, 2752) >= 8 * 2752 * 4
     assert ci.coreinfer_ffn_decode_stack_workspace_bytes(32, 1, 4096, 3277) >= 256 + 3 * 4096 * 4
+    assert ci.coreinfer_ffn_decode_stack_workspace_bytes(32, 8, 4096, 2752) >= 8 * 2752 * 4 + 3 * 8 * 4096 * 4
