@@ -195,3 +195,31 @@ def test_prefill_side_stream_gives_the_same_sets_and_weights():
     for a, b in zip(ref, got):
         for u, v in zip(a, b):
             assert u.tobytes() == v.tobytes()
+
+
+def test_full_size_gated_stack_of_eight_sequences():
+    """The ReLU-Llama-2-7B-shaped stack (32 gated layers, K = 2752) for 8 sequences sharing the
+    core sets, in one stack call: sampled layers against the oracle on the inputs they consumed."""
+    require_gpu()
+    cfg = wl.CONFIGS["relu-llama2-7b"]
+    B, L, d = 8, cfg.L, cfg.d_model
+    K = ci.coreinfer_count(cfg.beta, cfg.d_ff)
+    layers = [wl.compacted_weights_random(cfg, l, K, device="cuda") for l in range(L)]
+    arr = ci.binding.make_layers([(u, g, dn, None, None) for (u, g, dn) in layers])
+    x0 = wl.decode_input(cfg, 0, device="cuda", batch=B)
+    ws = torch.empty(ci.coreinfer_ffn_decode_stack_workspace_bytes(L, B, d, K), dtype=torch.uint8, device="cuda")
+    y_last = torch.empty((B, d), device="cuda")
+    y_layers = torch.empty((L, B, d), device="cuda")
+    x_layers = torch.empty((L, B, d), dtype=torch.bfloat16, device="cuda")
+    ci.coreinfer_ffn_decode_stack(arr, x0, ci.FFN_RELU_GATED, y_last, y_layers, x_layers, ws)
+    ci.coreinfer_workspace_status(ws)
+    assert torch.isfinite(y_layers).all()
+    assert torch.equal(y_last, y_layers[L - 1])
+    for l in (0, 17, 31):
+        up, gate, down = layers[l]
+        y_o = oracle.ffn(to_f32_np(x_layers[l]), ci.FFN_RELU_GATED, to_f32_np(up), to_f32_np(gate), to_f32_np(down))
+        assert_ffn_close(y_layers[l].cpu().numpy(), y_o, torch.bfloat16)
+        if l + 1 < L:
+            for b in (0, 7):
+                x_next = torch.from_numpy(oracle.glue(to_f32_np(x_layers[l])[b], y_layers[l][b].cpu().numpy())).to(torch.bfloat16)
+                np.testing.assert_allclose(to_f32_np(x_layers[l + 1])[b], x_next.float().numpy(), rtol=2 ** -7, atol=2 ** -7)
