@@ -408,8 +408,11 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
             }
             __syncthreads();
         }
+        // When the whole bin is admitted (need == eq_total) its remaining bits do not matter: every
+        // entry at or above the bin's lowest pattern is a member, and the search stops early.
+        // After the second digit most bins hold a single entry, so the third pass is rare.
 #pragma unroll 1
-        for (int pass = 1; pass < 3 && need > 0; ++pass) {
+        for (int pass = 1; pass < 3 && need > 0 && need != eq_total; ++pass) {
             const int shift = pass == 1 ? 11 : 0;
             const uint32_t dmask = pass == 1 ? 0xFFFu : 0x7FFu;
             const int pshift = pass == 1 ? 23 : 11;                   // prefix = bits >> pshift
