@@ -438,10 +438,13 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
         if (need == 0) {
             // no positive entry in this row: nothing to count
         } else if (need == eq_total) {
+            // masked entries are 0; after an early stop in the subnormal bin vstar is 0 too, and
+            // the smallest positive pattern, 1, is the bin's lower bound
+            const uint32_t lo = vstar ? vstar : 1u;
 #pragma unroll
-            for (int i = 0; i < VPT; ++i)     // vstar > 0, masked entries are 0
-                cnt8[i] += (held[i].x >= vstar ? 1u : 0u) | (held[i].y >= vstar ? 0x100u : 0u) |
-                           (held[i].z >= vstar ? 0x10000u : 0u) | (held[i].w >= vstar ? 0x1000000u : 0u);
+            for (int i = 0; i < VPT; ++i)
+                cnt8[i] += (held[i].x >= lo ? 1u : 0u) | (held[i].y >= lo ? 0x100u : 0u) |
+                           (held[i].z >= lo ? 0x10000u : 0u) | (held[i].w >= lo ? 0x1000000u : 0u);
         } else {
             // more entries equal the threshold than places left: lower index first.
             // Index order = vector round i, then thread, then element.
