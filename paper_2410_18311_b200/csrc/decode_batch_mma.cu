@@ -304,7 +304,6 @@ decode_batch_mma_kernel(const MmaParams p)
     // dacc[t]: columns j = jw + 16 t + lane / 4 (+ 8), sequences 2 (lane % 4) + {0, 1}.  Turn each tile
     // in this warp's scratch so that a lane owns 4 consecutive columns of one sequence.
     float* st = scratch + warp * 128;            // [8 sequences][16 columns]
-    float* stage = reinterpret_cast<float*>(ring);   // [B][d]: needs 2 B of the ring's slots
     named_bar_sync(1, kMmaThreads);              // the up phase's last use of the scratch is over
 #pragma unroll
     for (int t = 0; t < kMmaMaxTiles; ++t) {
@@ -323,20 +322,10 @@ decode_batch_mma_kernel(const MmaParams p)
                     v.x += __bfloat162float(p.bdown[j]);     v.y += __bfloat162float(p.bdown[j + 1]);
                     v.z += __bfloat162float(p.bdown[j + 2]); v.w += __bfloat162float(p.bdown[j + 3]);
                 }
-                *reinterpret_cast<float4*>(stage + (size_t)nn * p.d + j) = v;
+                red_add_v4(p.y + (size_t)nn * p.d + j, v.x, v.y, v.z, v.w);
             }
             __syncwarp();
         }
-    }
-    // The CTA's partial y [B][d] now sits where the ring was (every row has been consumed: the
-    // barrier above came after the last read).  It leaves as one bulk reduction per sequence
-    // instead of some eight thousand 16-byte reductions per CTA.
-    fence_proxy_async();
-    named_bar_sync(1, kMmaThreads);
-    if (tid == 0 && !*abort_flag) {
-        for (int b = 0; b < p.B; ++b)
-            bulk_reduce_add_f32(p.y + (size_t)b * p.d, smem_u32(stage + (size_t)b * p.d), (uint32_t)p.d * (uint32_t)sizeof(float));
-        bulk_wait_all();
     }
 }
 
