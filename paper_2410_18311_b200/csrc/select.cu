@@ -301,8 +301,7 @@ constexpr int kWarpHistStride = 257;     // 256 exponent bins; odd so that the w
 template <int VPT>
 __global__ void __launch_bounds__(kSelThreads, 1)
 select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long ld, double alpha,
-                        uint16_t* __restrict__ partial, int32_t* __restrict__ f_direct,
-                        unsigned* __restrict__ status, int row_bytes)
+                        uint16_t* __restrict__ partial, unsigned* __restrict__ status, int row_bytes)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     const int buf_bytes = (row_bytes + 127) & ~127;
@@ -479,29 +478,6 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
             if (clock64() - t0 > kSelWaitCycles) { atomicMax(status, (unsigned)kStatusTimeout); break; }
     }
 
-    if (f_direct) {
-        // Eq. 3 finished here: the CTA's counters go into the row buffer as 32-bit words and the
-        // copy engine adds them into f (zeroed by the host on this stream) in L2; no partial rows
-        // and no second kernel.
-        __syncthreads();                               // the last copy into the buffer has landed
-        uint4* cs = reinterpret_cast<uint4*>(smem);
-#pragma unroll
-        for (int i = 0; i < VPT; ++i) {
-            const int v = tid + i * kSelThreads;
-            if (v < nvec) cs[v] = make_uint4(cnt8[i] & 0xffu, (cnt8[i] >> 8) & 0xffu, (cnt8[i] >> 16) & 0xffu, cnt8[i] >> 24);
-        }
-        fence_proxy_async();
-        __syncthreads();
-        if (tid == 0 && !sh->abort_flag) {
-            const uint32_t whole = (uint32_t)(N / 4) * 16u;    // f has exactly N entries
-            for (uint32_t off = 0; off < whole; off += kCopyChunk)
-                bulk_reduce_add_u32(reinterpret_cast<unsigned*>(f_direct) + off / 4, smem_u32(smem) + off,
-                                    min(kCopyChunk, whole - off));
-            for (int n = (N / 4) * 4; n < N; ++n) atomicAdd(&f_direct[n], reinterpret_cast<const int*>(smem)[n]);
-            bulk_wait_all();                           // the buffer must outlive the engine's reads
-        }
-        return;
-    }
     uint16_t* out = partial + (size_t)blockIdx.x * ((size_t)nvec * 4);
 #pragma unroll
     for (int i = 0; i < VPT; ++i) {
@@ -655,12 +631,12 @@ static size_t sel_fast_fixed_smem()
 
 template <int VPT>
 static coreinfer_status launch_rows_fast(int grid, size_t smem, cudaStream_t st, const float* act, int T, int N,
-                                         long long ld, double alpha, uint16_t* partial, int32_t* f_direct,
-                                         unsigned* status, int row_bytes)
+                                         long long ld, double alpha, uint16_t* partial, unsigned* status,
+                                         int row_bytes)
 {
     auto kern = select_rows_fast_kernel<VPT>;
     CI_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    kern<<<grid, kSelThreads, smem, st>>>(act, T, N, ld, alpha, partial, f_direct, status, row_bytes);
+    kern<<<grid, kSelThreads, smem, st>>>(act, T, N, ld, alpha, partial, status, row_bytes);
     CI_CUDA(cudaGetLastError());
     return COREINFER_OK;
 }
@@ -676,7 +652,7 @@ size_t coreinfer_select_workspace_bytes(int32_t T, int32_t d_ff)
     if (T < 1 || d_ff < 1) return 0;
     const size_t n4 = ((size_t)d_ff + 3) & ~(size_t)3;
     const size_t ctas = (size_t)(T < kSelMaxCtas ? T : kSelMaxCtas);
-    return kSelCtrlBytes + ((ctas * n4 * sizeof(uint16_t) + 15) & ~(size_t)15) + n4 * sizeof(int32_t);
+    return kSelCtrlBytes + ctas * n4 * sizeof(uint16_t) + n4 * sizeof(int32_t);
 }
 
 coreinfer_status coreinfer_select_core(const void* act, coreinfer_dtype act_dtype, int32_t T, int32_t d_ff,
@@ -719,8 +695,7 @@ coreinfer_status coreinfer_select_core(const void* act, coreinfer_dtype act_dtyp
 
     unsigned* status = (unsigned*)workspace;
     uint16_t* partial = (uint16_t*)((uint8_t*)workspace + kSelCtrlBytes);
-    int32_t* f = counts_out ? counts_out
-                            : (int32_t*)((uint8_t*)partial + (((size_t)(T < kSelMaxCtas ? T : kSelMaxCtas) * n4 * sizeof(uint16_t) + 15) & ~(size_t)15));
+    int32_t* f = counts_out ? counts_out : (int32_t*)(partial + (size_t)(T < kSelMaxCtas ? T : kSelMaxCtas) * n4);
     CI_CUDA(cudaMemsetAsync(workspace, 0, kSelCtrlBytes, st));
 
     const size_t fixed = sel_fixed_smem();
@@ -729,14 +704,11 @@ coreinfer_status coreinfer_select_core(const void* act, coreinfer_dtype act_dtyp
     const int nbuf = (fixed + 2 * buf <= (size_t)di.smem_optin) ? 2 : 1;
     const size_t smem = fixed + nbuf * buf;
     const size_t smem_fast = sel_fast_fixed_smem() + buf;
-    // the fast kernel's CTAs add their counters straight into f (bulk reductions need 16-byte alignment)
-    const bool direct = fast && aligned16(f);
-    if (direct) CI_CUDA(cudaMemsetAsync(f, 0, (size_t)d_ff * sizeof(int32_t), st));
     const int vpt = (n4 / 4 + kSelThreads - 1) / kSelThreads;
 #define CI_ROWS(V)                                                                                        \
     case V:                                                                                               \
         s = fast ? launch_rows_fast<V>(G, smem_fast, st, (const float*)act, T, d_ff, (long long)ld_act,   \
-                                       alpha, partial, direct ? f : nullptr, status, row_bytes)           \
+                                       alpha, partial, status, row_bytes)                                 \
                  : launch_rows<V>(G, smem, st, (const float*)act, T, d_ff, (long long)ld_act, alpha,      \
                                   partial, status, nbuf, row_bytes);                                      \
         break;
@@ -747,10 +719,8 @@ coreinfer_status coreinfer_select_core(const void* act, coreinfer_dtype act_dtyp
 #undef CI_ROWS
     if (s != COREINFER_OK) return s;
 
-    if (!direct) {
-        select_count_kernel<<<(n4 / 4 + kCountCols - 1) / kCountCols, kCountCols * kCountSlices, 0, st>>>(partial, G, n4, d_ff, f);
-        CI_CUDA(cudaGetLastError());
-    }
+    select_count_kernel<<<(n4 / 4 + kCountCols - 1) / kCountCols, kCountCols * kCountSlices, 0, st>>>(partial, G, n4, d_ff, f);
+    CI_CUDA(cudaGetLastError());
 
     size_t smem_top = ((size_t)n4 + n4 / 32 + 8) * sizeof(int) + kSelBins * sizeof(int) + sizeof(SelShared) + 16;
     int top_shift = 0;
