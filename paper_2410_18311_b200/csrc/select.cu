@@ -48,11 +48,9 @@ struct SelShared {
     int abort_flag;
 };
 
-// Exclusive prefix sum over the block's NT threads; *total gets the block sum.
-template <int NT = kSelThreads>
+// Exclusive prefix sum over the block's threads; *total gets the block sum.
 __device__ __forceinline__ int block_excl_scan(int v, SelShared* sh, int* total)
 {
-    constexpr int NW = NT / 32;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     int incl = v;
 #pragma unroll
@@ -63,17 +61,17 @@ __device__ __forceinline__ int block_excl_scan(int v, SelShared* sh, int* total)
     if (lane == 31) sh->warp_tot[warp] = incl;
     __syncthreads();
     if (warp == 0) {
-        int w = lane < NW ? sh->warp_tot[lane] : 0;
+        int w = sh->warp_tot[lane];
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             int t = __shfl_up_sync(0xffffffffu, w, o);
             if (lane >= o) w += t;
         }
-        if (lane < NW) sh->warp_tot[lane] = w;
+        sh->warp_tot[lane] = w;
     }
     __syncthreads();
     const int base = warp > 0 ? sh->warp_tot[warp - 1] : 0;
-    *total = sh->warp_tot[NW - 1];
+    *total = sh->warp_tot[kSelWarps - 1];
     __syncthreads();
     return base + incl - v;
 }
@@ -82,17 +80,16 @@ __device__ __forceinline__ int block_excl_scan(int v, SelShared* sh, int* total)
 // (1 <= k <= total): sh->bin, sh->above = elements in higher bins, sh->bin_count.
 // With k_from_total, k = ceil(alpha * total) is formed here (total = number of positives).
 // Returns k (block-uniform); with k == 0 nothing else is written.
-template <int NT = kSelThreads>
 __device__ __forceinline__ int find_bin(const int* hist, int k, bool k_from_total, double alpha,
                                         SelShared* sh)
 {
-    constexpr int PER = kSelBins / NT;            // bins per thread (4 with 1024 threads), walked from the top
+    constexpr int PER = kSelBins / kSelThreads;   // 4 bins per thread, walked from the top
     const int top = kSelBins - 1 - PER * (int)threadIdx.x;
     int c[PER], s = 0;
 #pragma unroll
     for (int i = 0; i < PER; ++i) { c[i] = hist[top - i]; s += c[i]; }
     int total;
-    const int before = block_excl_scan<NT>(s, sh, &total);
+    const int before = block_excl_scan(s, sh, &total);
     if (k_from_total) k = count_dev(alpha, total);
     if (k > 0 && before < k && k <= before + s) {
         int above = before;
@@ -301,18 +298,16 @@ select_rows_kernel(const float* __restrict__ act, int T, int N, long long ld, do
 //    that are left spread evenly.
 constexpr int kWarpHistStride = 257;     // 256 exponent bins; odd so that the warps' copies of a bin use different banks
 
-// NT threads per CTA: 1024 (one CTA per SM), or 512 for narrow rows, where two CTAs share an SM
-// and work on two rows at once.
-template <int NT, int VPT>
-__global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1)
+template <int VPT>
+__global__ void __launch_bounds__(kSelThreads, 1)
 select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long ld, double alpha,
                         uint16_t* __restrict__ partial, unsigned* __restrict__ status, int row_bytes)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     const int buf_bytes = (row_bytes + 127) & ~127;
     int* hist = reinterpret_cast<int*>(smem + buf_bytes);                        // [kSelBins]
-    int* whist = hist + kSelBins;                                                // [(NT / 32)][kWarpHistStride]
-    uint64_t* bar = reinterpret_cast<uint64_t*>(whist + (((NT / 32) * kWarpHistStride + 1) & ~1));
+    int* whist = hist + kSelBins;                                                // [kSelWarps][kWarpHistStride]
+    uint64_t* bar = reinterpret_cast<uint64_t*>(whist + ((kSelWarps * kWarpHistStride + 1) & ~1));
     SelShared* sh = reinterpret_cast<SelShared*>(bar + 1);
 
     const int tid = threadIdx.x;
@@ -369,7 +364,7 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
         uint4 held[VPT];
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
-            const int v = tid + i * NT;
+            const int v = tid + i * kSelThreads;
             uint4 q = make_uint4(0, 0, 0, 0);
             if (v < nvec) q = row[v];
             if (v * 4 + 0 >= N || !is_pos_bits(q.x)) q.x = 0u;
@@ -379,7 +374,7 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
             held[i] = q;
         }
         // per-warp exponent histograms start at zero (their last use ended before the barrier above)
-        for (int i = tid; i < (NT / 32) * kWarpHistStride; i += NT) whist[i] = 0;
+        for (int i = tid; i < kSelWarps * kWarpHistStride; i += kSelThreads) whist[i] = 0;
         __syncthreads();             // every thread holds its columns: the buffer may be refilled
         if (tid == 0 && t + G < T) issue_row(t + G);
 
@@ -396,16 +391,16 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
                     if (bb[e] != 0u) atomicAdd(&mine[bb[e] >> 23], 1);
             }
             __syncthreads();
-            for (int b = tid; b < kSelBins; b += NT) {
+            for (int b = tid; b < kSelBins; b += kSelThreads) {
                 int c = 0;
                 if (b < 256) {
 #pragma unroll 8
-                    for (int w = 0; w < (NT / 32); ++w) c += whist[w * kWarpHistStride + b];
+                    for (int w = 0; w < kSelWarps; ++w) c += whist[w * kWarpHistStride + b];
                 }
                 hist[b] = c;
             }
             __syncthreads();
-            need = find_bin<NT>(hist, 0, true, alpha, sh);
+            need = find_bin(hist, 0, true, alpha, sh);
             if (need > 0) {
                 vstar = (uint32_t)sh->bin << 23;
                 need -= sh->above;
@@ -421,7 +416,7 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
             const int shift = pass == 1 ? 11 : 0;
             const uint32_t dmask = pass == 1 ? 0xFFFu : 0x7FFu;
             const int pshift = pass == 1 ? 23 : 11;                   // prefix = bits >> pshift
-            for (int i = tid; i < kSelBins; i += NT) hist[i] = 0;
+            for (int i = tid; i < kSelBins; i += kSelThreads) hist[i] = 0;
             __syncthreads();
 #pragma unroll
             for (int i = 0; i < VPT; ++i) {
@@ -432,7 +427,7 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
                         atomicAdd(&hist[(bb[e] >> shift) & dmask], 1);
             }
             __syncthreads();
-            need = find_bin<NT>(hist, need, false, alpha, sh);
+            need = find_bin(hist, need, false, alpha, sh);
             vstar |= (uint32_t)sh->bin << shift;
             need -= sh->above;
             eq_total = sh->bin_count;
@@ -461,7 +456,7 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
 #pragma unroll
                 for (int e = 0; e < 4; ++e) c += (bb[e] == vstar) ? 1 : 0;
                 int tot;
-                int rank = taken + block_excl_scan<NT>(c, sh, &tot);
+                int rank = taken + block_excl_scan(c, sh, &tot);
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     if (bb[e] > vstar) cnt8[i] += 1u << (8 * e);
@@ -486,7 +481,7 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
     uint16_t* out = partial + (size_t)blockIdx.x * ((size_t)nvec * 4);
 #pragma unroll
     for (int i = 0; i < VPT; ++i) {
-        const int v = tid + i * NT;
+        const int v = tid + i * kSelThreads;
         if (v < nvec) {
             uint2 w;
             w.x = (cnt8[i] & 0xffu) | ((cnt8[i] & 0xff00u) << 8);
@@ -628,20 +623,20 @@ static coreinfer_status launch_rows(int grid, size_t smem, cudaStream_t st, cons
     return COREINFER_OK;
 }
 
-static size_t sel_fast_fixed_smem(int nt = kSelThreads)
+static size_t sel_fast_fixed_smem()
 {
-    return kSelBins * sizeof(int) + (((nt / 32) * kWarpHistStride + 1) & ~1) * sizeof(int) + sizeof(uint64_t) +
+    return kSelBins * sizeof(int) + ((kSelWarps * kWarpHistStride + 1) & ~1) * sizeof(int) + sizeof(uint64_t) +
            sizeof(SelShared) + 128;
 }
 
-template <int NT, int VPT>
+template <int VPT>
 static coreinfer_status launch_rows_fast(int grid, size_t smem, cudaStream_t st, const float* act, int T, int N,
                                          long long ld, double alpha, uint16_t* partial, unsigned* status,
                                          int row_bytes)
 {
-    auto kern = select_rows_fast_kernel<NT, VPT>;
+    auto kern = select_rows_fast_kernel<VPT>;
     CI_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    kern<<<grid, NT, smem, st>>>(act, T, N, ld, alpha, partial, status, row_bytes);
+    kern<<<grid, kSelThreads, smem, st>>>(act, T, N, ld, alpha, partial, status, row_bytes);
     CI_CUDA(cudaGetLastError());
     return COREINFER_OK;
 }
@@ -694,17 +689,6 @@ coreinfer_status coreinfer_select_core(const void* act, coreinfer_dtype act_dtyp
     if ((T + G_fast - 1) / G_fast > 255) G_fast = (T + 254) / 255;
     const bool fast = G_fast <= kSelMaxCtas && sel_fast_fixed_smem() + buf <= (size_t)di.smem_optin;
     if (fast) G = G_fast;
-    // Narrow rows (at most 8 vectors per thread with 512 threads) and more rows than SMs: two
-    // CTAs of 512 threads per SM work on two rows at once (a row's selection is a chain of
-    // barriers and shared-memory atomics that leaves most of the SM idle).
-    const int vpt_half = (n4 / 4 + 511) / 512;
-    const size_t smem_half = sel_fast_fixed_smem(512) + buf;
-    const bool half = fast && vpt_half <= 8 && T > di.sm_count && 2 * (smem_half + 1024) <= (size_t)228 * 1024;
-    if (half) {
-        G = T < 2 * di.sm_count ? T : 2 * di.sm_count;
-        if (G > kSelMaxCtas) G = kSelMaxCtas;
-        if ((T + G - 1) / G > 255) G = (T + 254) / 255;       // <= kSelMaxCtas, as for G_fast
-    }
     if ((T + G - 1) / G > 65535)
         CI_FAIL(COREINFER_ERR_UNSUPPORTED, "T = %d: more than 65535 rows per CTA", T);
     const int K = coreinfer_count(beta, d_ff);
@@ -723,30 +707,16 @@ coreinfer_status coreinfer_select_core(const void* act, coreinfer_dtype act_dtyp
     const int vpt = (n4 / 4 + kSelThreads - 1) / kSelThreads;
 #define CI_ROWS(V)                                                                                        \
     case V:                                                                                               \
-        s = fast ? launch_rows_fast<1024, V>(G, smem_fast, st, (const float*)act, T, d_ff,                \
-                                             (long long)ld_act, alpha, partial, status, row_bytes)        \
+        s = fast ? launch_rows_fast<V>(G, smem_fast, st, (const float*)act, T, d_ff, (long long)ld_act,   \
+                                       alpha, partial, status, row_bytes)                                 \
                  : launch_rows<V>(G, smem, st, (const float*)act, T, d_ff, (long long)ld_act, alpha,      \
                                   partial, status, nbuf, row_bytes);                                      \
         break;
-#define CI_ROWS_HALF(V)                                                                                   \
-    case V:                                                                                               \
-        s = launch_rows_fast<512, V>(G, smem_half, st, (const float*)act, T, d_ff, (long long)ld_act,     \
-                                     alpha, partial, status, row_bytes);                                  \
-        break;
-    if (half) {
-        switch (vpt_half) {
-            CI_ROWS_HALF(1) CI_ROWS_HALF(2) CI_ROWS_HALF(3) CI_ROWS_HALF(4) CI_ROWS_HALF(5) CI_ROWS_HALF(6)
-            CI_ROWS_HALF(7) CI_ROWS_HALF(8)
-            default: CI_FAIL(COREINFER_ERR_UNSUPPORTED, "d_ff = %d not built", d_ff);
-        }
-    } else {
-        switch (vpt) {
-            CI_ROWS(1) CI_ROWS(2) CI_ROWS(3) CI_ROWS(4) CI_ROWS(5) CI_ROWS(6) CI_ROWS(7) CI_ROWS(8) CI_ROWS(9)
-            default: CI_FAIL(COREINFER_ERR_UNSUPPORTED, "d_ff = %d not built", d_ff);
-        }
+    switch (vpt) {
+        CI_ROWS(1) CI_ROWS(2) CI_ROWS(3) CI_ROWS(4) CI_ROWS(5) CI_ROWS(6) CI_ROWS(7) CI_ROWS(8) CI_ROWS(9)
+        default: CI_FAIL(COREINFER_ERR_UNSUPPORTED, "d_ff = %d not built", d_ff);
     }
 #undef CI_ROWS
-#undef CI_ROWS_HALF
     if (s != COREINFER_OK) return s;
 
     select_count_kernel<<<(n4 / 4 + kCountCols - 1) / kCountCols, kCountCols * kCountSlices, 0, st>>>(partial, G, n4, d_ff, f);
