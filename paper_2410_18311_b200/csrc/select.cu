@@ -381,20 +381,16 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
         // ---- radix select of the k-th largest positive pattern: 8 + 12 + 11 bits ----
         uint32_t vstar = 0u;
         int need = 0, eq_total = 0;
-        {   // Exponent digit.  Shared-memory atomic instructions are what this kernel runs out of,
-            // so only a quarter of the entries (the first of every vector) go into the histogram;
-            // the bin that sample points to is then verified on all entries with two counts
-            // (entries in higher bins, entries in the bin), and moved by one bin at a time while
-            // it is wrong: the result is exact, the sample only decides where the search starts.
+        {   // exponent digit
             int* mine = whist + (tid >> 5) * kWarpHistStride;
-            int pc = 0;
 #pragma unroll
             for (int i = 0; i < VPT; ++i) {
-                pc += (held[i].x != 0u) + (held[i].y != 0u) + (held[i].z != 0u) + (held[i].w != 0u);
-                if (held[i].x != 0u) atomicAdd(&mine[held[i].x >> 23], 1);
+                const uint32_t bb[4] = {held[i].x, held[i].y, held[i].z, held[i].w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (bb[e] != 0u) atomicAdd(&mine[bb[e] >> 23], 1);
             }
-            int P;                                     // positives of the row
-            block_excl_scan(pc, sh, &P);
+            __syncthreads();
             for (int b = tid; b < kSelBins; b += kSelThreads) {
                 int c = 0;
                 if (b < 256) {
@@ -404,35 +400,11 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
                 hist[b] = c;
             }
             __syncthreads();
-            const int k = count_dev(alpha, P);
-            if (k > 0) {
-                const int ks = find_bin(hist, 0, true, (double)k / (double)P, sh);   // the same rank in the sample
-                int e = ks > 0 ? sh->bin : 127;
-                __syncthreads();
-                unsigned A = 0, C = 0;
-                for (int it = 0; it < 512; ++it) {
-                    const uint32_t lo = (uint32_t)e << 23, hi = (uint32_t)(e + 1) << 23;   // hi = 2^31 for e = 255: nothing is above
-                    unsigned a = 0, c = 0;
-#pragma unroll
-                    for (int i = 0; i < VPT; ++i) {
-                        const uint32_t bb[4] = {held[i].x, held[i].y, held[i].z, held[i].w};
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            a += bb[q] >= hi ? 1u : 0u;
-                            c += (bb[q] >= lo && bb[q] < hi && bb[q] != 0u) ? 1u : 0u;
-                        }
-                    }
-                    int tot;                           // both counts in one scan: each stays below 2^16
-                    block_excl_scan((int)((a << 16) | c), sh, &tot);
-                    A = (unsigned)tot >> 16;
-                    C = (unsigned)tot & 0xffffu;
-                    if ((unsigned)k <= A) { if (e == 255) break; ++e; }
-                    else if ((unsigned)k > A + C) { if (e == 0) break; --e; }
-                    else break;
-                }
-                vstar = (uint32_t)e << 23;
-                need = k - (int)A;
-                eq_total = (int)C;
+            need = find_bin(hist, 0, true, alpha, sh);
+            if (need > 0) {
+                vstar = (uint32_t)sh->bin << 23;
+                need -= sh->above;
+                eq_total = sh->bin_count;
             }
             __syncthreads();
         }
