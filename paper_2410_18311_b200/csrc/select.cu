@@ -319,6 +319,8 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
         sh->abort_flag = 0;
         mbar_fence_init();
     }
+    // the per-warp exponent histograms start at zero; every row's merge leaves them at zero again
+    for (int i = tid; i < kSelWarps * kWarpHistStride; i += kSelThreads) whist[i] = 0;
     __syncthreads();
 
     int issued = 0;                        // thread 0: copies issued
@@ -373,15 +375,15 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
             if (v * 4 + 3 >= N || !is_pos_bits(q.w)) q.w = 0u;
             held[i] = q;
         }
-        // per-warp exponent histograms start at zero (their last use ended before the barrier above)
-        for (int i = tid; i < kSelWarps * kWarpHistStride; i += kSelThreads) whist[i] = 0;
         __syncthreads();             // every thread holds its columns: the buffer may be refilled
         if (tid == 0 && t + G < T) issue_row(t + G);
+        // the shared histogram of the second digit starts at zero (the exponent digit does not use it)
+        for (int i = tid; i < kSelBins; i += kSelThreads) hist[i] = 0;
 
         // ---- radix select of the k-th largest positive pattern: 8 + 12 + 11 bits ----
         uint32_t vstar = 0u;
         int need = 0, eq_total = 0;
-        {   // exponent digit
+        {   // exponent digit: per-warp histograms, merged and searched by the first 256 threads
             int* mine = whist + (tid >> 5) * kWarpHistStride;
 #pragma unroll
             for (int i = 0; i < VPT; ++i) {
@@ -391,22 +393,26 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
                     if (bb[e] != 0u) atomicAdd(&mine[bb[e] >> 23], 1);
             }
             __syncthreads();
-            for (int b = tid; b < kSelBins; b += kSelThreads) {
-                int c = 0;
-                if (b < 256) {
+            // thread t < 256 merges bin 255 - t (so thread order is bin order from the top) and
+            // leaves the per-warp words at zero for the next row
+            int c = 0;
+            if (tid < 256) {
 #pragma unroll 8
-                    for (int w = 0; w < kSelWarps; ++w) c += whist[w * kWarpHistStride + b];
+                for (int w = 0; w < kSelWarps; ++w) {
+                    c += whist[w * kWarpHistStride + 255 - tid];
+                    whist[w * kWarpHistStride + 255 - tid] = 0;
                 }
-                hist[b] = c;
             }
+            int total;                                 // positives of the row
+            const int before = block_excl_scan(c, sh, &total);
+            const int k = count_dev(alpha, total);
+            if (k > 0 && before < k && k <= before + c) { sh->bin = 255 - tid; sh->above = before; sh->bin_count = c; }
             __syncthreads();
-            need = find_bin(hist, 0, true, alpha, sh);
-            if (need > 0) {
+            if (k > 0) {
                 vstar = (uint32_t)sh->bin << 23;
-                need -= sh->above;
+                need = k - sh->above;
                 eq_total = sh->bin_count;
             }
-            __syncthreads();
         }
         // When the whole bin is admitted (need == eq_total) its remaining bits do not matter: every
         // entry at or above the bin's lowest pattern is a member, and the search stops early.
@@ -416,8 +422,10 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
             const int shift = pass == 1 ? 11 : 0;
             const uint32_t dmask = pass == 1 ? 0xFFFu : 0x7FFu;
             const int pshift = pass == 1 ? 23 : 11;                   // prefix = bits >> pshift
-            for (int i = tid; i < kSelBins; i += kSelThreads) hist[i] = 0;
-            __syncthreads();
+            if (pass == 2) {                                          // rare: the histogram is used a second time
+                for (int i = tid; i < kSelBins; i += kSelThreads) hist[i] = 0;
+                __syncthreads();
+            }
 #pragma unroll
             for (int i = 0; i < VPT; ++i) {
                 const uint32_t bb[4] = {held[i].x, held[i].y, held[i].z, held[i].w};
@@ -427,11 +435,10 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
                         atomicAdd(&hist[(bb[e] >> shift) & dmask], 1);
             }
             __syncthreads();
-            need = find_bin(hist, need, false, alpha, sh);
+            need = find_bin(hist, need, false, alpha, sh);            // ends with a barrier: the result is published
             vstar |= (uint32_t)sh->bin << shift;
             need -= sh->above;
             eq_total = sh->bin_count;
-            __syncthreads();
         }
 
         // ---- membership (Eq. 1) and its count (Eq. 3) ----
@@ -465,7 +472,7 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
                 taken += tot;
             }
         }
-        __syncthreads();   // the shared scratch is free again
+        // no barrier here: the next row writes shared memory only after its own barriers
     }
 
     // Never leave with a copy into this CTA's shared memory in flight.  On the normal path
