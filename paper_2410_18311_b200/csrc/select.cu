@@ -369,11 +369,20 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
             const int v = tid + i * kSelThreads;
             uint4 q = make_uint4(0, 0, 0, 0);
             if (v < nvec) q = row[v];
-            if (v * 4 + 0 >= N || !is_pos_bits(q.x)) q.x = 0u;
-            if (v * 4 + 1 >= N || !is_pos_bits(q.y)) q.y = 0u;
-            if (v * 4 + 2 >= N || !is_pos_bits(q.z)) q.z = 0u;
-            if (v * 4 + 3 >= N || !is_pos_bits(q.w)) q.w = 0u;
+            q.x = is_pos_bits(q.x) ? q.x : 0u;
+            q.y = is_pos_bits(q.y) ? q.y : 0u;
+            q.z = is_pos_bits(q.z) ? q.z : 0u;
+            q.w = is_pos_bits(q.w) ? q.w : 0u;
             held[i] = q;
+        }
+        if (N & 3) {                                   // ragged width: the row's last vector reaches beyond d_ff
+#pragma unroll
+            for (int i = 0; i < VPT; ++i) {
+                const int v = tid + i * kSelThreads;
+                if (v * 4 + 1 >= N) held[i].y = 0u;
+                if (v * 4 + 2 >= N) held[i].z = 0u;
+                if (v * 4 + 3 >= N) held[i].w = 0u;
+            }
         }
         __syncthreads();             // every thread holds its columns: the buffer may be refilled
         if (tid == 0 && t + G < T) issue_row(t + G);
@@ -384,13 +393,13 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
         uint32_t vstar = 0u;
         int need = 0, eq_total = 0;
         {   // exponent digit: per-warp histograms, merged and searched by the first 256 threads
-            int* mine = whist + (tid >> 5) * kWarpHistStride;
+            const uint32_t mine = smem_u32(whist + (tid >> 5) * kWarpHistStride);
 #pragma unroll
             for (int i = 0; i < VPT; ++i) {
-                const uint32_t bb[4] = {held[i].x, held[i].y, held[i].z, held[i].w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    if (bb[e] != 0u) atomicAdd(&mine[bb[e] >> 23], 1);
+                red_shared_inc_if_nonzero(mine + ((held[i].x >> 23) << 2), held[i].x);
+                red_shared_inc_if_nonzero(mine + ((held[i].y >> 23) << 2), held[i].y);
+                red_shared_inc_if_nonzero(mine + ((held[i].z >> 23) << 2), held[i].z);
+                red_shared_inc_if_nonzero(mine + ((held[i].w >> 23) << 2), held[i].w);
             }
             __syncthreads();
             // thread t < 256 merges bin 255 - t (so thread order is bin order from the top) and
@@ -426,13 +435,18 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
                 for (int i = tid; i < kSelBins; i += kSelThreads) hist[i] = 0;
                 __syncthreads();
             }
+            {   // entries whose higher digits equal the threshold's: lo <= bits < lo + span (0 is "masked")
+                const uint32_t base = (vstar >> pshift) << pshift;
+                const uint32_t lo = base ? base : 1u;
+                const uint32_t span = base + (1u << pshift) - lo;
+                const uint32_t hist_s = smem_u32(hist);
 #pragma unroll
-            for (int i = 0; i < VPT; ++i) {
-                const uint32_t bb[4] = {held[i].x, held[i].y, held[i].z, held[i].w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    if (bb[e] != 0u && (bb[e] >> pshift) == (vstar >> pshift))
-                        atomicAdd(&hist[(bb[e] >> shift) & dmask], 1);
+                for (int i = 0; i < VPT; ++i) {
+                    red_shared_inc_if_in_range(hist_s + (((held[i].x >> shift) & dmask) << 2), held[i].x, lo, span);
+                    red_shared_inc_if_in_range(hist_s + (((held[i].y >> shift) & dmask) << 2), held[i].y, lo, span);
+                    red_shared_inc_if_in_range(hist_s + (((held[i].z >> shift) & dmask) << 2), held[i].z, lo, span);
+                    red_shared_inc_if_in_range(hist_s + (((held[i].w >> shift) & dmask) << 2), held[i].w, lo, span);
+                }
             }
             __syncthreads();
             need = find_bin(hist, need, false, alpha, sh);            // ends with a barrier: the result is published
