@@ -108,18 +108,10 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
         : "memory");
 }
 
-// Predicated shared-memory increments by 32-bit shared-window address (no branch, no generic
-// address conversion): add 1 at `addr` if v != 0 / if (v - lo) < span (unsigned).
-__device__ __forceinline__ void red_shared_inc_if_nonzero(uint32_t addr, uint32_t v)
+// Shared-memory increment by 32-bit shared-window address (no generic address conversion).
+__device__ __forceinline__ void red_shared_inc(uint32_t addr)
 {
-    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %1, 0;\n\t@q red.shared.add.u32 [%0], 1;\n\t}"
-                 ::"r"(addr), "r"(v) : "memory");
-}
-__device__ __forceinline__ void red_shared_inc_if_in_range(uint32_t addr, uint32_t v, uint32_t lo, uint32_t span)
-{
-    asm volatile("{\n\t.reg .pred q;\n\t.reg .u32 t;\n\tsub.u32 t, %1, %2;\n\tsetp.lt.u32 q, t, %3;\n\t"
-                 "@q red.shared.add.u32 [%0], 1;\n\t}"
-                 ::"r"(addr), "r"(v), "r"(lo), "r"(span) : "memory");
+    asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(addr) : "memory");
 }
 
 __device__ __forceinline__ void named_bar_sync(int id, int nthreads)

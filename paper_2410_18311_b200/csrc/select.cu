@@ -296,7 +296,7 @@ select_rows_kernel(const float* __restrict__ act, int T, int N, long long ld, do
 //    crowd into a handful of exponents: in one shared histogram those additions queue on the
 //    same few words), then 12 and 11 mantissa bits in the shared histogram, where the entries
 //    that are left spread evenly.
-constexpr int kWarpHistStride = 257;     // 256 exponent bins; odd so that the warps' copies of a bin use different banks
+constexpr int kWarpHistStride = 288;     // 256 exponent bins + 32 words (one per lane) that take the increments of masked entries
 
 template <int VPT>
 __global__ void __launch_bounds__(kSelThreads, 1)
@@ -305,8 +305,8 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
 {
     extern __shared__ __align__(128) uint8_t smem[];
     const int buf_bytes = (row_bytes + 127) & ~127;
-    int* hist = reinterpret_cast<int*>(smem + buf_bytes);                        // [kSelBins]
-    int* whist = hist + kSelBins;                                                // [kSelWarps][kWarpHistStride]
+    int* hist = reinterpret_cast<int*>(smem + buf_bytes);                        // [kSelBins + 32]: bins, then one word per lane for entries that do not count
+    int* whist = hist + kSelBins + 32;                                           // [kSelWarps][kWarpHistStride]
     uint64_t* bar = reinterpret_cast<uint64_t*>(whist + ((kSelWarps * kWarpHistStride + 1) & ~1));
     SelShared* sh = reinterpret_cast<SelShared*>(bar + 1);
 
@@ -393,13 +393,16 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
         uint32_t vstar = 0u;
         int need = 0, eq_total = 0;
         {   // exponent digit: per-warp histograms, merged and searched by the first 256 threads
+            // Every entry increments a word: its exponent's bin, or (masked entries) this lane's own
+            // spare word, so that the loop has no branch (a predicated atomic compiles to one).
             const uint32_t mine = smem_u32(whist + (tid >> 5) * kWarpHistStride);
+            const uint32_t spare = 256u + (uint32_t)(tid & 31);
 #pragma unroll
             for (int i = 0; i < VPT; ++i) {
-                red_shared_inc_if_nonzero(mine + ((held[i].x >> 23) << 2), held[i].x);
-                red_shared_inc_if_nonzero(mine + ((held[i].y >> 23) << 2), held[i].y);
-                red_shared_inc_if_nonzero(mine + ((held[i].z >> 23) << 2), held[i].z);
-                red_shared_inc_if_nonzero(mine + ((held[i].w >> 23) << 2), held[i].w);
+                red_shared_inc(mine + ((held[i].x ? held[i].x >> 23 : spare) << 2));
+                red_shared_inc(mine + ((held[i].y ? held[i].y >> 23 : spare) << 2));
+                red_shared_inc(mine + ((held[i].z ? held[i].z >> 23 : spare) << 2));
+                red_shared_inc(mine + ((held[i].w ? held[i].w >> 23 : spare) << 2));
             }
             __syncthreads();
             // thread t < 256 merges bin 255 - t (so thread order is bin order from the top) and
@@ -440,12 +443,14 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
                 const uint32_t lo = base ? base : 1u;
                 const uint32_t span = base + (1u << pshift) - lo;
                 const uint32_t hist_s = smem_u32(hist);
+                const uint32_t spare = (uint32_t)kSelBins + (uint32_t)(tid & 31);      // this lane's word for the others
+                auto word_of = [&](uint32_t b) { return hist_s + (((b - lo) < span ? ((b >> shift) & dmask) : spare) << 2); };
 #pragma unroll
                 for (int i = 0; i < VPT; ++i) {
-                    red_shared_inc_if_in_range(hist_s + (((held[i].x >> shift) & dmask) << 2), held[i].x, lo, span);
-                    red_shared_inc_if_in_range(hist_s + (((held[i].y >> shift) & dmask) << 2), held[i].y, lo, span);
-                    red_shared_inc_if_in_range(hist_s + (((held[i].z >> shift) & dmask) << 2), held[i].z, lo, span);
-                    red_shared_inc_if_in_range(hist_s + (((held[i].w >> shift) & dmask) << 2), held[i].w, lo, span);
+                    red_shared_inc(word_of(held[i].x));
+                    red_shared_inc(word_of(held[i].y));
+                    red_shared_inc(word_of(held[i].z));
+                    red_shared_inc(word_of(held[i].w));
                 }
             }
             __syncthreads();
@@ -646,7 +651,7 @@ static coreinfer_status launch_rows(int grid, size_t smem, cudaStream_t st, cons
 
 static size_t sel_fast_fixed_smem()
 {
-    return kSelBins * sizeof(int) + ((kSelWarps * kWarpHistStride + 1) & ~1) * sizeof(int) + sizeof(uint64_t) +
+    return (kSelBins + 32) * sizeof(int) + ((kSelWarps * kWarpHistStride + 1) & ~1) * sizeof(int) + sizeof(uint64_t) +
            sizeof(SelShared) + 128;
 }
 
