@@ -361,7 +361,11 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
         __syncthreads();
         if (sh->abort_flag) break;   // block-uniform
 
-        // this thread's columns; 0 stands for "not positive" (or beyond d_ff)
+        // This thread's columns.  kMasked (sign bit alone) stands for "not positive" (or beyond
+        // d_ff): its "exponent" is 256, one past the real bins, it is below every positive pattern
+        // as a signed integer and far from all of them as an unsigned difference, so no loop below
+        // needs a test for it.
+        constexpr uint32_t kMasked = 0x80000000u;
         const uint4* row = reinterpret_cast<const uint4*>(smem);
         uint4 held[VPT];
 #pragma unroll
@@ -369,19 +373,19 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
             const int v = tid + i * kSelThreads;
             uint4 q = make_uint4(0, 0, 0, 0);
             if (v < nvec) q = row[v];
-            q.x = is_pos_bits(q.x) ? q.x : 0u;
-            q.y = is_pos_bits(q.y) ? q.y : 0u;
-            q.z = is_pos_bits(q.z) ? q.z : 0u;
-            q.w = is_pos_bits(q.w) ? q.w : 0u;
+            q.x = is_pos_bits(q.x) ? q.x : kMasked;
+            q.y = is_pos_bits(q.y) ? q.y : kMasked;
+            q.z = is_pos_bits(q.z) ? q.z : kMasked;
+            q.w = is_pos_bits(q.w) ? q.w : kMasked;
             held[i] = q;
         }
         if (N & 3) {                                   // ragged width: the row's last vector reaches beyond d_ff
 #pragma unroll
             for (int i = 0; i < VPT; ++i) {
                 const int v = tid + i * kSelThreads;
-                if (v * 4 + 1 >= N) held[i].y = 0u;
-                if (v * 4 + 2 >= N) held[i].z = 0u;
-                if (v * 4 + 3 >= N) held[i].w = 0u;
+                if (v * 4 + 1 >= N) held[i].y = kMasked;
+                if (v * 4 + 2 >= N) held[i].z = kMasked;
+                if (v * 4 + 3 >= N) held[i].w = kMasked;
             }
         }
         __syncthreads();             // every thread holds its columns: the buffer may be refilled
@@ -393,16 +397,15 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
         uint32_t vstar = 0u;
         int need = 0, eq_total = 0;
         {   // exponent digit: per-warp histograms, merged and searched by the first 256 threads
-            // Every entry increments a word: its exponent's bin, or (masked entries) this lane's own
-            // spare word, so that the loop has no branch (a predicated atomic compiles to one).
+            // Every entry increments a word, its exponent's bin (masked entries: word 256, never
+            // read), so the loop has neither test nor branch (a predicated atomic compiles to one).
             const uint32_t mine = smem_u32(whist + (tid >> 5) * kWarpHistStride);
-            const uint32_t spare = 256u + (uint32_t)(tid & 31);
 #pragma unroll
             for (int i = 0; i < VPT; ++i) {
-                red_shared_inc(mine + ((held[i].x ? held[i].x >> 23 : spare) << 2));
-                red_shared_inc(mine + ((held[i].y ? held[i].y >> 23 : spare) << 2));
-                red_shared_inc(mine + ((held[i].z ? held[i].z >> 23 : spare) << 2));
-                red_shared_inc(mine + ((held[i].w ? held[i].w >> 23 : spare) << 2));
+                red_shared_inc(mine + ((held[i].x >> 23) << 2));
+                red_shared_inc(mine + ((held[i].y >> 23) << 2));
+                red_shared_inc(mine + ((held[i].z >> 23) << 2));
+                red_shared_inc(mine + ((held[i].w >> 23) << 2));
             }
             __syncthreads();
             // thread t < 256 merges bin 255 - t (so thread order is bin order from the top) and
@@ -438,13 +441,15 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
                 for (int i = tid; i < kSelBins; i += kSelThreads) hist[i] = 0;
                 __syncthreads();
             }
-            {   // entries whose higher digits equal the threshold's: lo <= bits < lo + span (0 is "masked")
+            {   // entries whose higher digits equal the threshold's have bits - base < 2^pshift; their
+                // digit is that difference's; everything else lands in the word after the bins
                 const uint32_t base = (vstar >> pshift) << pshift;
-                const uint32_t lo = base ? base : 1u;
-                const uint32_t span = base + (1u << pshift) - lo;
                 const uint32_t hist_s = smem_u32(hist);
-                const uint32_t spare = (uint32_t)kSelBins + (uint32_t)(tid & 31);      // this lane's word for the others
-                auto word_of = [&](uint32_t b) { return hist_s + (((b - lo) < span ? ((b >> shift) & dmask) : spare) << 2); };
+                const uint32_t nbins = dmask + 1u;
+                auto word_of = [&](uint32_t b) {
+                    const uint32_t dgt = (b - base) >> shift;
+                    return hist_s + ((dgt < nbins ? dgt : (uint32_t)kSelBins) << 2);
+                };
 #pragma unroll
                 for (int i = 0; i < VPT; ++i) {
                     red_shared_inc(word_of(held[i].x));
@@ -464,13 +469,12 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
         if (need == 0) {
             // no positive entry in this row: nothing to count
         } else if (need == eq_total) {
-            // masked entries are 0; after an early stop in the subnormal bin vstar is 0 too, and
-            // the smallest positive pattern, 1, is the bin's lower bound
-            const uint32_t lo = vstar ? vstar : 1u;
+            // signed comparison: masked entries are the most negative integer, positives are positive
+            const int lo = (int)vstar;
 #pragma unroll
             for (int i = 0; i < VPT; ++i)
-                cnt8[i] += (held[i].x >= lo ? 1u : 0u) | (held[i].y >= lo ? 0x100u : 0u) |
-                           (held[i].z >= lo ? 0x10000u : 0u) | (held[i].w >= lo ? 0x1000000u : 0u);
+                cnt8[i] += ((int)held[i].x >= lo ? 1u : 0u) | ((int)held[i].y >= lo ? 0x100u : 0u) |
+                           ((int)held[i].z >= lo ? 0x10000u : 0u) | ((int)held[i].w >= lo ? 0x1000000u : 0u);
         } else {
             // more entries equal the threshold than places left: lower index first.
             // Index order = vector round i, then thread, then element.
@@ -485,7 +489,7 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
                 int rank = taken + block_excl_scan(c, sh, &tot);
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    if (bb[e] > vstar) cnt8[i] += 1u << (8 * e);
+                    if ((int)bb[e] > (int)vstar) cnt8[i] += 1u << (8 * e);
                     else if (bb[e] == vstar) { cnt8[i] += (rank < need ? 1u : 0u) << (8 * e); ++rank; }
                 }
                 taken += tot;
