@@ -48,6 +48,7 @@ def parse_args():
                     help="profiling target: only decode launches through the first LAYERS layers of the config "
                          "on random compacted weights (small enough for an ncu capture); prints a short JSON line")
     ap.add_argument("--tokens", type=int, default=2, help="decode launches per step in --decode-only mode")
+    ap.add_argument("--batch", type=int, default=1, help="sequences per decode step in --decode-only mode (1..8)")
     return ap.parse_args()
 
 
@@ -485,14 +486,15 @@ def run_decode_only(args, cfg):
     layers = [wl.compacted_weights_random(cfg, l, K, device="cuda") for l in range(cfg.L)]
     arr = ci.binding.make_layers([(u, g, dn, None, None) for (u, g, dn) in layers])
     kind = ci.FFN_RELU_GATED if cfg.gated else ci.FFN_RELU
-    xs = torch.cat([wl.decode_input(cfg, s, device="cuda") for s in range(args.tokens)], dim=0)
-    ys = torch.empty((args.tokens, cfg.d_model), device="cuda")
-    ws = torch.empty(ci.coreinfer_ffn_decode_stack_workspace_bytes(cfg.L, 1, cfg.d_model, K), dtype=torch.uint8,
+    B = args.batch
+    xs = torch.stack([wl.decode_input(cfg, s, device="cuda", batch=B) for s in range(args.tokens)], dim=0)
+    ys = torch.empty((args.tokens, B, cfg.d_model), device="cuda")
+    ws = torch.empty(ci.coreinfer_ffn_decode_stack_workspace_bytes(cfg.L, B, cfg.d_model, K), dtype=torch.uint8,
                      device="cuda")
 
     def step():
         for t in range(args.tokens):
-            ci.coreinfer_ffn_decode_stack(arr, xs[t:t + 1], kind, ys[t:t + 1], None, None, ws)
+            ci.coreinfer_ffn_decode_stack(arr, xs[t], kind, ys[t], None, None, ws)
     for _ in range(args.warmup):
         step()
     torch.cuda.synchronize()
@@ -505,8 +507,9 @@ def run_decode_only(args, cfg):
     ci.coreinfer_workspace_status(ws)
     us = e0.elapsed_time(e1) * 1e3 / (args.steps * args.tokens)
     nbytes = cfg.L * cfg.n_mat * K * cfg.d_model * cfg.esize
-    print(json.dumps({"mode": "decode-only", "workload": cfg.name, "layers": cfg.L, "K": K, "us_per_launch": us,
-                      "bytes_per_launch": nbytes, "gbs": nbytes / us / 1e3}), flush=True)
+    print(json.dumps({"mode": "decode-only", "workload": cfg.name, "layers": cfg.L, "K": K, "batch": B,
+                      "us_per_launch": us, "us_per_layer": us / cfg.L, "bytes_per_launch": nbytes,
+                      "gbs": nbytes / us / 1e3, "sequence_tokens_per_s": B * 1e6 / us}), flush=True)
 
 
 def main():

@@ -16,6 +16,11 @@
 //         [d_model / 16 columns] x [8 sequences] accumulators stay in registers for the slab.
 //   out:  tiles are turned in shared memory and added to y with vector reductions.
 // Every wait is bounded as in the batch-1 kernel.
+//
+// Inside the multi-layer stack the launches are chained with programmatic dependent launch: a
+// CTA of the next layer's kernel starts as soon as an SM is free, and its producer warp streams
+// that layer's weights (which depend on nothing) into the ring while the previous layer's last
+// CTAs and the glue kernel finish; only the consumers wait for the layer input.
 #include "common.cuh"
 
 namespace coreinfer {
@@ -96,6 +101,7 @@ decode_batch_mma_kernel(const MmaParams p)
     const int n_up_units = (n + RU - 1) / RU;
     const int n_dn_units = (n + 15) / 16;
 
+    grid_dep_launch_dependents();     // the next launch of a chain may start filling free SMs
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) {
             mbar_init(smem_u32(&full_bar[s]), 1);
@@ -164,6 +170,10 @@ decode_batch_mma_kernel(const MmaParams p)
     const int JW = p.d / kMmaWarps;                   // columns of this warp (a multiple of 16)
     const int jw = warp * JW;
     const int ntile = JW / 16;                        // <= kMmaMaxTiles
+
+    // In a chain x (and the cleared y) come from the launch before this one: wait for it here.
+    // The producer warp does not wait: it reads weights only.
+    grid_dep_wait();
 
     // x^T fragments: B[k][n] = x[n][jw + 16 t + k]; lane holds k = 2 (lane % 4) + {0, 1} (+ 8), n = lane / 4
     uint32_t xb[kMmaMaxTiles][2];
@@ -330,8 +340,11 @@ decode_batch_mma_kernel(const MmaParams p)
 }
 
 // Returns COREINFER_ERR_UNSUPPORTED (without setting an error text) when the shape is not built here.
+// chained = false: y is cleared here and the launch is an ordinary one.  chained = true (inside
+// the stack): y has been cleared by an earlier operation of the stream, and the launch may start
+// before the kernel launched before it on the stream has finished (its consumers wait for it).
 coreinfer_status decode_batched_mma(const void* x, int batch, bool gated, int d_model, const coreinfer_layer& ly,
-                                    float* y, unsigned* status, const DeviceInfo& di, cudaStream_t st)
+                                    float* y, unsigned* status, const DeviceInfo& di, cudaStream_t st, bool chained)
 {
     if (d_model % (kMmaWarps * 16) != 0 || d_model / (kMmaWarps * 16) > kMmaMaxTiles) return COREINFER_ERR_UNSUPPORTED;
     MmaParams p;
@@ -359,16 +372,32 @@ coreinfer_status decode_batched_mma(const void* x, int batch, bool gated, int d_
     if (slots < 17) return COREINFER_ERR_UNSUPPORTED;
     p.n_slots = (int)slots;
     const size_t smem = fixed + (size_t)p.n_slots * p.slot_stride;
-    CI_CUDA(cudaMemsetAsync(y, 0, (size_t)batch * d_model * sizeof(float), st));
-    if (gated) {
-        CI_CUDA(cudaFuncSetAttribute(decode_batch_mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        decode_batch_mma_kernel<true><<<G, kMmaBlock, smem, st>>>(p);
-    } else {
-        CI_CUDA(cudaFuncSetAttribute(decode_batch_mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        decode_batch_mma_kernel<false><<<G, kMmaBlock, smem, st>>>(p);
-    }
-    CI_CUDA(cudaGetLastError());
+    if (!chained) CI_CUDA(cudaMemsetAsync(y, 0, (size_t)batch * d_model * sizeof(float), st));
+    auto kern = gated ? decode_batch_mma_kernel<true> : decode_batch_mma_kernel<false>;
+    CI_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)G);
+    cfg.blockDim = dim3((unsigned)kMmaBlock);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = chained ? 1 : 0;
+    CI_CUDA(cudaLaunchKernelEx(&cfg, kern, p));
     return COREINFER_OK;
+}
+
+// Whether decode_batched_mma serves this shape (same conditions as above).
+bool decode_batched_mma_serves(int d_model, int K, const DeviceInfo& di)
+{
+    if (d_model % (kMmaWarps * 16) != 0 || d_model / (kMmaWarps * 16) > kMmaMaxTiles) return false;
+    const size_t stride = (size_t)d_model * 2 + 16;
+    const int rmax = (K + di.sm_count - 1) / di.sm_count + 1;
+    const size_t fixed = stride + 2 * kMmaMaxSlots * sizeof(uint64_t) + kMmaWarps * 128 * sizeof(float)
+                         + (size_t)3 * 8 * ((rmax + 15) & ~15) * sizeof(__nv_bfloat16) + 16 + 128;
+    return ((long long)di.smem_optin - (long long)fixed) / (long long)stride >= 17;
 }
 
 }  // namespace coreinfer

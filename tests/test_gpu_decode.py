@@ -156,6 +156,7 @@ def test_stack_of_small_batches_teacher_forced(B):
                     np.testing.assert_allclose(xl[l + 1][b], x_next, rtol=tol, atol=tol)
         # without the per-layer dumps the result is the same up to the order of the sums
         y2 = torch.empty((B, d), device="cuda")
+        ws.fill_(0xFF)      # NaN patterns: a y buffer of the workspace that nobody cleared would show
         ci.coreinfer_ffn_decode_stack(arr, x0.cuda(), kind, y2, None, None, ws)
         ci.coreinfer_workspace_status(ws)
         from helpers import rel_err_rms
