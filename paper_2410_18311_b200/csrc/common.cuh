@@ -158,19 +158,6 @@ __device__ __forceinline__ void bulk_wait_all()
     asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
 
-// Programmatic dependent launch.  launch_dependents: the next kernel of the stream, if it was
-// launched with programmatic stream serialization, may start once every CTA of this grid has
-// executed this (or exited).  wait: returns when the kernels this grid depends on have completed
-// and their writes are visible; without such a dependency it returns at once.
-__device__ __forceinline__ void grid_dep_launch_dependents()
-{
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-}
-__device__ __forceinline__ void grid_dep_wait()
-{
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-}
-
 #endif  // __CUDACC__
 
 }  // namespace coreinfer

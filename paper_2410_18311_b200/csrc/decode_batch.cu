@@ -177,8 +177,11 @@ static coreinfer_status run_t(int batch, const void* x, bool gated, int d_model,
 
 // decode_batch_mma.cu: tensor-core kernel for bf16 rows of up to 4096 columns
 coreinfer_status decode_batched_mma(const void* x, int batch, bool gated, int d_model, const coreinfer_layer& ly,
-                                    float* y, unsigned* status, const DeviceInfo& di, cudaStream_t st, bool chained);
+                                    float* y, unsigned* status, const DeviceInfo& di, cudaStream_t st);
 bool decode_batched_mma_serves(int d_model, int K, const DeviceInfo& di);
+coreinfer_status decode_stack_batched_mma(const coreinfer_layer* layers, int L, const void* x0, int batch, bool gated,
+                                          int d_model, float* y_last, float* y_layers, void* x_layers, float* ybuf,
+                                          unsigned* ctrl, const DeviceInfo& di, cudaStream_t st);
 
 coreinfer_status decode_batched(const void* x, int batch, coreinfer_dtype dtype, coreinfer_ffn_kind kind,
                                 int d_model, const coreinfer_layer& ly, float* y, void* workspace,
@@ -190,7 +193,7 @@ coreinfer_status decode_batched(const void* x, int batch, coreinfer_dtype dtype,
     const bool gated = kind == COREINFER_FFN_RELU_GATED;
     if (clear_status) CI_CUDA(cudaMemsetAsync(workspace, 0, kCtrlBytesB, st));   // status word
     if (dtype == COREINFER_BF16) {
-        s = decode_batched_mma(x, batch, gated, d_model, ly, y, (unsigned*)workspace, di, st, false);
+        s = decode_batched_mma(x, batch, gated, d_model, ly, y, (unsigned*)workspace, di, st);
         if (s != COREINFER_ERR_UNSUPPORTED) return s;          // otherwise: shape not built there, use the plain kernels
     }
     float* h = (float*)((uint8_t*)workspace + kCtrlBytesB);
@@ -205,22 +208,15 @@ template <typename T> static __device__ __forceinline__ T from_f(float v);
 template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
-// Glue between two layers, one CTA per sequence: x_next = round((x + y) / rms(x + y)), the same
-// formula (rsqrtf of the mean square) as in the batch-1 stack kernel.  y_clear, when given, is
-// the buffer the next layer adds into: each CTA clears its sequence's row of it.
-// In a chain of dependent launches the kernel lets its successor start at once and itself waits
-// for its predecessor (the FFN kernel that produced y) before it touches global memory.
+// Glue between two layers for the per-layer path, one CTA per sequence: x_next = round((x + y) /
+// rms(x + y)), the same formula (rsqrtf of the mean square) as in the batch-1 stack kernel.
 template <typename T>
 __global__ void __launch_bounds__(256)
 batch_glue_kernel(const T* __restrict__ x, const float* __restrict__ y, T* __restrict__ x_next,
-                  T* __restrict__ x_dump, float* __restrict__ y_clear, int d, float inv_d)
+                  T* __restrict__ x_dump, int d, float inv_d)
 {
     __shared__ float part[8];
-    grid_dep_launch_dependents();
-    grid_dep_wait();
     const size_t base = (size_t)blockIdx.x * d;
-    if (y_clear)
-        for (int j = threadIdx.x; j < d; j += 256) y_clear[base + j] = 0.f;
     float ss = 0.f;
     for (int j = threadIdx.x; j < d; j += 256) {
         const float v = to_f(x[base + j]) + y[base + j];
@@ -242,40 +238,18 @@ batch_glue_kernel(const T* __restrict__ x, const float* __restrict__ y, T* __res
     }
 }
 
-template <typename T>
-static coreinfer_status launch_glue(const void* x, const float* y, void* x_next, void* x_dump, float* y_clear,
-                                    int batch, int d_model, bool chained, cudaStream_t st)
-{
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)batch);
-    cfg.blockDim = dim3(256);
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = chained ? 1 : 0;
-    CI_CUDA(cudaLaunchKernelEx(&cfg, batch_glue_kernel<T>, (const T*)x, y, (T*)x_next, (T*)x_dump, y_clear, d_model,
-                               1.0f / (float)d_model));
-    return COREINFER_OK;
-}
-
 static size_t align256(size_t b) { return (b + 255) & ~(size_t)255; }
 
-// layer scratch (status word + h) | two y buffers (ping-pong) | two x buffers (ping-pong)
+// layer scratch (status word + h) | three y buffers | two x buffers (ping-pong)
 size_t decode_stack_batched_workspace_bytes(int batch, int d_model, int K_max)
 {
-    return align256(kCtrlBytesB + (size_t)batch * K_max * sizeof(float)) + 4 * align256((size_t)batch * d_model * sizeof(float));
+    return align256(kCtrlBytesB + (size_t)batch * K_max * sizeof(float)) + 5 * align256((size_t)batch * d_model * sizeof(float));
 }
 
-// The stack for 2..8 sequences: per layer one batched FFN (every weight byte read once for all
-// sequences) and one glue launch.  Outputs as in the batch-1 stack: y_layers / x_layers
-// [L][batch][d_model] when given.
-//
-// Where the tensor-core kernel serves every layer, the 2 L - 1 launches form one chain of
-// programmatic dependent launches with nothing else in between: every y the chain adds into is
-// cleared before it starts or by the glue kernel one layer ahead, so a layer's kernel is resident
-// and streaming its weights while the layer before it drains.
+// The stack for 2..8 sequences.  Outputs as in the batch-1 stack: y_layers / x_layers
+// [L][batch][d_model] when given.  Where the tensor-core kernel serves every layer the whole
+// stack is one persistent launch (decode_batch_mma.cu); otherwise per layer one batched FFN call
+// and one glue launch.
 coreinfer_status decode_stack_batched(const coreinfer_layer* layers, int L, const void* x0, int batch,
                                       coreinfer_dtype dtype, coreinfer_ffn_kind kind, int d_model, float* y_last,
                                       float* y_layers, void* x_layers, void* workspace, size_t workspace_bytes,
@@ -292,38 +266,40 @@ coreinfer_status decode_stack_batched(const coreinfer_layer* layers, int L, cons
     const size_t ybytes = align256(row * sizeof(float));
     uint8_t* w = (uint8_t*)workspace;
     uint8_t* y0 = w + align256(kCtrlBytesB + (size_t)batch * Kmax * sizeof(float));
-    float* ybuf[2] = {(float*)y0, (float*)(y0 + ybytes)};
-    uint8_t* xbuf[2] = {y0 + 2 * ybytes, y0 + 3 * ybytes};
+    float* ybuf = (float*)y0;                                    // three buffers, ybytes apart
+    uint8_t* xbuf[2] = {y0 + 3 * ybytes, y0 + 4 * ybytes};
     const bool gated = kind == COREINFER_FFN_RELU_GATED;
 
     DeviceInfo di;
     coreinfer_status s = device_info(&di);
     if (s != COREINFER_OK) return s;
-    bool chain = dtype == COREINFER_BF16;
-    for (int l = 0; l < L && chain; ++l) chain = decode_batched_mma_serves(d_model, layers[l].K, di);
+    bool one_launch = dtype == COREINFER_BF16 && ybytes == row * sizeof(float);
+    for (int l = 0; l < L && one_launch; ++l) one_launch = decode_batched_mma_serves(d_model, layers[l].K, di);
 
-    CI_CUDA(cudaMemsetAsync(workspace, 0, kCtrlBytesB, st));      // status word: sticky over the layers
+    CI_CUDA(cudaMemsetAsync(workspace, 0, kCtrlBytesB, st));      // status word (sticky over the layers), barrier counter
     if (x_layers) CI_CUDA(cudaMemcpyAsync(x_layers, x0, row * esize, cudaMemcpyDeviceToDevice, st));
-    auto y_of = [&](int l) -> float* {
-        return y_layers ? y_layers + (size_t)l * row : (l == L - 1 ? y_last : ybuf[l & 1]);
-    };
-    if (chain) {
-        // everything the chain adds into before a glue kernel could have cleared it
-        if (y_layers) {
-            CI_CUDA(cudaMemsetAsync(y_layers, 0, (size_t)L * row * sizeof(float), st));
-        } else {
-            CI_CUDA(cudaMemsetAsync(y_last, 0, row * sizeof(float), st));
-            if (L > 1) CI_CUDA(cudaMemsetAsync(ybuf[0], 0, row * sizeof(float), st));
+
+    if (one_launch) {
+        // what the kernel adds into before it can have cleared it itself
+        if (y_layers) CI_CUDA(cudaMemsetAsync(y_layers, 0, (size_t)L * row * sizeof(float), st));
+        CI_CUDA(cudaMemsetAsync(y_last, 0, row * sizeof(float), st));
+        CI_CUDA(cudaMemsetAsync(ybuf, 0, 2 * ybytes, st));
+        s = decode_stack_batched_mma(layers, L, x0, batch, gated, d_model, y_last, y_layers, x_layers, ybuf,
+                                     (unsigned*)workspace, di, st);
+        if (s != COREINFER_ERR_UNSUPPORTED) {
+            if (s != COREINFER_OK) return s;
+            if (y_layers)
+                CI_CUDA(cudaMemcpyAsync(y_last, y_layers + (size_t)(L - 1) * row, row * sizeof(float),
+                                        cudaMemcpyDeviceToDevice, st));
+            return COREINFER_OK;
         }
     }
+
     const void* x_in = x0;
     for (int l = 0; l < L; ++l) {
         const bool last = (l == L - 1);
-        float* y_out = y_of(l);
-        if (chain)
-            s = decode_batched_mma(x_in, batch, gated, d_model, layers[l], y_out, (unsigned*)workspace, di, st, l > 0);
-        else
-            s = decode_batched(x_in, batch, dtype, kind, d_model, layers[l], y_out, workspace, st, false);
+        float* y_out = y_layers ? y_layers + (size_t)l * row : (last ? y_last : ybuf);
+        s = decode_batched(x_in, batch, dtype, kind, d_model, layers[l], y_out, workspace, st, false);
         if (s != COREINFER_OK) return s;
         if (last) {
             if (y_out != y_last) CI_CUDA(cudaMemcpyAsync(y_last, y_out, row * sizeof(float), cudaMemcpyDeviceToDevice, st));
@@ -331,12 +307,13 @@ coreinfer_status decode_stack_batched(const coreinfer_layer* layers, int L, cons
         }
         void* x_next = xbuf[l & 1];
         void* dump = x_layers ? (void*)((uint8_t*)x_layers + (size_t)(l + 1) * row * esize) : nullptr;
-        // in a chain the glue kernel clears what the next layer adds into, unless that was done up front
-        float* y_clear = (chain && !y_layers && l + 1 < L - 1) ? ybuf[(l + 1) & 1] : nullptr;
-        s = dtype == COREINFER_BF16
-                ? launch_glue<__nv_bfloat16>(x_in, y_out, x_next, dump, y_clear, batch, d_model, chain, st)
-                : launch_glue<float>(x_in, y_out, x_next, dump, y_clear, batch, d_model, false, st);
-        if (s != COREINFER_OK) return s;
+        if (dtype == COREINFER_BF16)
+            batch_glue_kernel<__nv_bfloat16><<<batch, 256, 0, st>>>((const __nv_bfloat16*)x_in, y_out, (__nv_bfloat16*)x_next,
+                                                                   (__nv_bfloat16*)dump, d_model, 1.0f / (float)d_model);
+        else
+            batch_glue_kernel<float><<<batch, 256, 0, st>>>((const float*)x_in, y_out, (float*)x_next, (float*)dump,
+                                                           d_model, 1.0f / (float)d_model);
+        CI_CUDA(cudaGetLastError());
         x_in = x_next;
     }
     return COREINFER_OK;
