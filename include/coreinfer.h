@@ -158,8 +158,10 @@ coreinfer_status coreinfer_ffn_decode(const void* x, int32_t batch, coreinfer_dt
  *              consumed, or NULL.
  *   workspace  at least coreinfer_ffn_decode_stack_workspace_bytes().
  * 1 <= batch <= COREINFER_MAX_BATCH, 1 <= L <= COREINFER_MAX_LAYERS.  batch 1 is the single
- * persistent launch described here; 2..8 sequences (sharing the core sets) run as one batched
- * FFN launch plus one glue launch per layer, every weight byte read once for all sequences.
+ * persistent launch described here; 2..8 sequences (sharing the core sets) read every weight
+ * byte once for all sequences: in bf16 with d_model a multiple of 256 up to 4096 again as one
+ * persistent launch (tensor cores, the sequences on the N side), otherwise as one batched FFN
+ * launch plus one glue launch per layer.
  * Thread blocks of this launch wait on one another at layer boundaries; every
  * such wait is bounded, and a wait that gives up makes all blocks return early
  * and records COREINFER_ERR_TIMEOUT in the workspace (read it with
