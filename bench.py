@@ -49,6 +49,9 @@ def parse_args():
                          "on random compacted weights (small enough for an ncu capture); prints a short JSON line")
     ap.add_argument("--tokens", type=int, default=2, help="decode launches per step in --decode-only mode")
     ap.add_argument("--batch", type=int, default=1, help="sequences per decode step in --decode-only mode (1..8)")
+    ap.add_argument("--sequences", type=int, default=None,
+                    help="also time the compacted stack for this many sequences sharing the core sets (2..8; "
+                         "default: 8 for the gated Llama-shaped workload, which is specified at 1 and 8, else off)")
     return ap.parse_args()
 
 
@@ -433,6 +436,21 @@ def run_ours(args, cfg):
         except torch.OutOfMemoryError:
             dense = {"skipped": "not enough free HBM for a second, dense copy of the stack"}
 
+    # ---- the same compacted stack for several sequences that share the core sets ----
+    batched = None
+    n_seq = args.sequences if args.sequences is not None else (8 if cfg.gated else 0)
+    if n_seq > 1 and rank == 0:
+        nb, nstep = n_seq, 16
+        xb = wl.decode_input(cfg, 0, device=dev, batch=nb)
+        yb = torch.empty((nb, cfg.d_model), device=dev)
+        wsb = torch.empty(ci.coreinfer_ffn_decode_stack_workspace_bytes(cfg.L, nb, cfg.d_model, stack.K),
+                          dtype=torch.uint8, device=dev)
+        ms = time_call(lambda: [ci.coreinfer_ffn_decode_stack(stack.layers, xb, stack.kind, yb, None, None, wsb, stream)
+                                for _ in range(nstep)], reps=2) / nstep
+        ci.coreinfer_workspace_status(wsb)
+        batched = {"batch": nb, "ms_per_step": ms, "sequence_tok_s": nb / (ms * 1e-3),
+                   "gbs": stack.compacted_bytes_per_token() / (ms * 1e-3) / 1e9, "steps_timed": 2 * nstep}
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -456,7 +474,7 @@ def run_ours(args, cfg):
         "decode": {"tok_s": steps_tok / (decode_ms * 1e-3), "ms_per_token": decode_ms / steps_tok,
                    "gbs": achieved, "frac_of_8TBs": achieved / 8000.0},
         "select_ms_per_layer": sel_ms, "compact_ms_per_layer": cmp_ms, "prefill_ms_per_request": prefill_ms,
-        "dense": dense,
+        "dense": dense, "batched": batched,
         "roofline": {"bound": "hbm", "kernel": "decode_stack_kernel", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_source": "of " + peak_src,
                      "bytes_per_launch": bytes_tok, "launch_us": launch_s * 1e6,
