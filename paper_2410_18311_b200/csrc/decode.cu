@@ -26,6 +26,8 @@
 // copies in flight and returns.
 #include "common.cuh"
 
+#include <stdlib.h>
+
 namespace coreinfer {
 
 constexpr int kMaxSlots = 64;
@@ -215,8 +217,14 @@ __device__ __forceinline__ float warp_reduce8(const float (&v)[8], int lane)
 // ------------------------------------------------------------------- kernel --
 // Ring stream order of one CTA and one layer (producer and consumers walk it in lock step): for
 // each slab row k0 .. k1-1 its up row, then (gated) its gate row; after those, the down rows
-// k0 .. k1-1.  Within each of the two phases the items are cut into batches of BATCH; batch b
-// belongs to consumer group b % NG.
+// k0 .. k1-1.  Within each of the two phases the items are cut into batches of BATCH.  With two
+// consumer groups every batch takes BATCH ring slots, the last batch of a phase being filled up
+// with empty items (no copy: the producer completes their barrier by a plain arrival), and the
+// batches of the whole launch are dealt out in turn: batch number g of the launch belongs to
+// group g % NG and starts at ring position (g * BATCH) % slots.  The ring holds a multiple of
+// NG * BATCH slots, so a slot is read by the same group in every pass of the ring: a group that
+// tests a slot's barrier has itself consumed the slot's previous fill, and can therefore never
+// mistake the parity of a fill that is still in flight for that of the one it wants.
 template <typename T, int NG, int VPT, bool GATED>
 __global__ void __launch_bounds__(NG * kGroupThreads + 32, 1)
 decode_stack_kernel(const __grid_constant__ DecodeParams p)
@@ -227,6 +235,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
     constexpr int NMAT = GATED ? 2 : 1;
     constexpr int NC = NG * kGroupThreads;           // consumer threads
     constexpr int BATCH = batch_for(NG, VPT);        // ring items per batch
+    constexpr int PADB = NG > 1 ? BATCH : 1;         // a phase takes a multiple of PADB ring slots
     constexpr int FLUSH = 16 / BATCH;                // own up batches per cross-lane reduction (16 row sums)
 
     extern __shared__ __align__(128) uint8_t smem[];
@@ -274,7 +283,8 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
             slab_of(cta, G, l, ly.K, &k0, &k1);
             const int n = k1 - k0;
             const int n_up = n * NMAT;            // items of the up (+ gate) phase
-            const int total = n_up + n;           // + the down rows
+            const int p_up = (n_up + PADB - 1) / PADB * PADB;          // ring slots of that phase
+            const int total = p_up + (n + PADB - 1) / PADB * PADB;     // + those of the down rows
             for (int q0 = 0, cnt = 0; q0 < total; q0 += cnt) {
                 if (*abort_flag) break;
                 cnt = min(round_max, total - q0);
@@ -295,20 +305,24 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
                 }
                 if (lane < cnt) {
                     const int q = q0 + lane;
-                    const uint8_t* src;
+                    const uint8_t* src = nullptr;         // stays NULL for an empty item
                     if (q < n_up) {
                         const int row = k0 + q / NMAT;
                         src = ((GATED && (q % NMAT)) ? ly.gate : ly.up) + (size_t)row * p.row_bytes;
-                    } else {
-                        src = ly.down + (size_t)(k0 + q - n_up) * p.row_bytes;
+                    } else if (q >= p_up && q - p_up < n) {
+                        src = ly.down + (size_t)(k0 + q - p_up) * p.row_bytes;
                     }
                     int sl = slot0 + lane;
                     uint32_t ph = phase0;
                     if (sl >= NS) { sl -= NS; ph ^= 1u; }
                     if (wait_slot(smem_u32(&empty_bar[sl]), ph ^ 1u, abort_flag, p.ctrl)) {
                         const uint32_t fb = smem_u32(&full_bar[sl]);
-                        mbar_arrive_expect_tx(fb, (uint32_t)p.row_bytes);
-                        bulk_g2s(smem_u32(ring + (size_t)sl * p.slot_bytes), src, (uint32_t)p.row_bytes, fb);
+                        if (src) {
+                            mbar_arrive_expect_tx(fb, (uint32_t)p.row_bytes);
+                            bulk_g2s(smem_u32(ring + (size_t)sl * p.slot_bytes), src, (uint32_t)p.row_bytes, fb);
+                        } else {
+                            mbar_arrive(fb);
+                        }
                     }
                 }
                 __syncwarp();
@@ -356,19 +370,21 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
 
     int slot = 0;                 // ring position of the next item of the stream
     uint32_t phase = 0;
-    auto skip_n = [&](int n) {    // items that belong to the other group
+    int gbatch = 0;               // two groups: number, within the launch, of the current phase's first batch
+    auto skip_n = [&](int n) {    // ring slots that belong to the other group
         slot += n;
         if (slot >= NS) { slot -= NS; phase ^= 1u; }
     };
     // wait for the next n items, pull them into registers (q[j][i] = vector i of item j), free them
     auto fetch = [&](uint4 (&q)[BATCH][VPT], int n) {
+        const int held = NG > 1 ? BATCH : n;      // ring slots of this batch (two groups: empty items included)
         {
             // test all barriers of the batch back to back (the tests overlap); only if one is
             // not complete yet fall back to the bounded waits, one by one
             bool ready = true;
 #pragma unroll
             for (int j = 0; j < BATCH; ++j) {
-                int sl = slot + (j < n ? j : 0);
+                int sl = slot + (j < held ? j : 0);
                 uint32_t ph = phase;
                 if (sl >= NS) { sl -= NS; ph ^= 1u; }
                 ready &= mbar_try_wait(smem_u32(&full_bar[sl]), ph);
@@ -376,7 +392,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
             if (!ready) {
                 int sl = slot;
                 uint32_t ph = phase;
-                for (int j = 0; j < n; ++j) {
+                for (int j = 0; j < held; ++j) {
                     wait_slot(smem_u32(&full_bar[sl]), ph, abort_flag, p.ctrl);
                     if (++sl == NS) { sl = 0; ph ^= 1u; }
                 }
@@ -405,12 +421,12 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
             }
         }
         __syncwarp();
-        if (lane < n && !*abort_flag) {
+        if (lane < held && !*abort_flag) {
             int sl = slot + lane;
             if (sl >= NS) sl -= NS;
             mbar_arrive(smem_u32(&empty_bar[sl]));
         }
-        skip_n(n);
+        skip_n(held);
     };
 
     for (int l = 0; l < p.L; ++l) {
@@ -430,7 +446,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
             int first_b = 0;                      // first of them
             for (int b = 0; b < nb; ++b) {
                 const int cnt = min(BATCH, n_up - b * BATCH);
-                if (NG > 1 && (b % NG) != grp) { skip_n(cnt); continue; }
+                if (NG > 1 && ((gbatch + b) % NG) != grp) { skip_n(BATCH); continue; }
                 uint4 q[BATCH][VPT];
                 fetch(q, cnt);
                 if (own == 0) first_b = b;
@@ -470,6 +486,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
                     own = 0;
                 }
             }
+            gbatch += nb;
         }
         named_bar_sync(1, NC);
         for (int r = tid; r < nrows; r += NC) {
@@ -508,7 +525,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
             const int nb = (nrows + BATCH - 1) / BATCH;
             for (int b = 0; b < nb; ++b) {
                 const int cnt = min(BATCH, nrows - b * BATCH);
-                if (NG > 1 && (b % NG) != grp) { skip_n(cnt); continue; }
+                if (NG > 1 && ((gbatch + b) % NG) != grp) { skip_n(BATCH); continue; }
                 uint4 q[BATCH][VPT];
                 fetch(q, cnt);
 #pragma unroll
@@ -526,6 +543,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
                     }
                 }
             }
+            gbatch += nb;
         }
 
         // ----------------------------------------- cross-CTA sum of partial y --
@@ -697,6 +715,17 @@ static coreinfer_status launch_one(const DecodeParams& p, int grid, size_t smem,
     return COREINFER_OK;
 }
 
+// Debugging aid: COREINFER_RING_SLOTS=n in the environment (read once) caps the ring of the
+// batch-1 stack kernel at n slots, so that tests can make the ring wrap every few rows.
+static int ring_slots_cap()
+{
+    static const int cap = [] {
+        const char* e = getenv("COREINFER_RING_SLOTS");
+        return e ? atoi(e) : 0;
+    }();
+    return cap;
+}
+
 static int groups_for(int nv) { return nv <= 2 * kGroupThreads ? 2 : 1; }
 static int vpt_for(int nv)
 {
@@ -802,9 +831,14 @@ static coreinfer_status decode_stack_b1(const coreinfer_layer* layers, int L, co
         CI_FAIL(COREINFER_ERR_UNSUPPORTED, "K = %d, d_model = %d do not fit in shared memory", Kmax, d_model);
     long long slots = ((long long)di.smem_optin - (long long)fixed) / p.slot_bytes;
     if (slots > kMaxSlots) slots = kMaxSlots;
+    if (ring_slots_cap() > 0 && slots > ring_slots_cap()) slots = ring_slots_cap();
     // With two groups a slot must always come back to the same group (a group never waits on the
-    // other's items, so only then can it never be a full ring pass ahead of a barrier it tests).
-    if (groups == 2 && slots >= 2 * batch) slots -= slots % (2 * batch);
+    // other's items, so only then can it never be a full ring pass ahead of a barrier it tests):
+    // every batch takes `batch` slots and the ring holds a whole number of batch pairs.
+    if (groups == 2) slots -= slots % (2 * batch);
+    if (slots < (long long)groups * batch)
+        CI_FAIL(COREINFER_ERR_UNSUPPORTED, "the ring of %lld slots is smaller than %d batches of %d rows", slots,
+                groups, batch);
     p.n_slots = (int)slots;
     const size_t smem = fixed + (size_t)p.n_slots * p.slot_bytes;
     // Measured on the four model shapes: about 100 KB of the next layer requested ahead of the

@@ -696,6 +696,8 @@ coreinfer_status coreinfer_select_core(const void* act, coreinfer_dtype act_dtyp
     if (T < 1 || d_ff < 1) CI_FAIL(COREINFER_ERR_INVALID_ARG, "T = %d, d_ff = %d must be >= 1", T, d_ff);
     if (!(alpha > 0.0 && alpha <= 1.0) || !(beta > 0.0 && beta <= 1.0))
         CI_FAIL(COREINFER_ERR_INVALID_ARG, "alpha = %g, beta = %g must lie in (0, 1]", alpha, beta);
+    if (coreinfer_count(beta, d_ff) < 1)
+        CI_FAIL(COREINFER_ERR_INVALID_ARG, "beta = %g selects no neuron of d_ff = %d", beta, d_ff);
     if (ld_act < d_ff || (ld_act & 3) != 0 || !aligned16(act))
         CI_FAIL(COREINFER_ERR_INVALID_ARG, "act must be 16-byte aligned with ld_act >= d_ff and ld_act %% 4 == 0");
     if (d_ff > kSelMaxVpt * kSelThreads * 4)

@@ -81,3 +81,38 @@ def gpu_decode(x, kind, up_c, gate_c, down_c, bup_c=None, bdown=None):
     ci.coreinfer_ffn_decode(x, kind, up_c, gate_c, down_c, bup_c, bdown, y, ws)
     ci.coreinfer_workspace_status(ws)
     return y.cpu().numpy()
+
+
+def check_stack_teacher_forced(layers_gpu, x0, kind, dtype, layers_to_check=None, noalloc=False):
+    """One coreinfer_ffn_decode_stack call with per-layer dumps; every checked layer's output is
+    compared with the oracle on the very input that layer consumed (Section 4.2), and the step
+    between layers with the oracle's residual + RMS glue.  layers_gpu: [(up, gate | None, down,
+    b_up | None, b_down | None)] CUDA tensors; x0 [B, d] CUDA.  Returns (y_last, y_layers, x_layers)."""
+    import oracle
+    L, (B, d) = len(layers_gpu), x0.shape
+    Kmax = max(ly[0].shape[0] for ly in layers_gpu)
+    arr = ci.binding.make_layers(layers_gpu)
+    y_last = torch.full((B, d), float("nan"), device="cuda")
+    y_layers = torch.full((L, B, d), float("nan"), device="cuda")
+    x_layers = torch.zeros((L, B, d), dtype=dtype, device="cuda")
+    if noalloc:
+        ci.coreinfer_ffn_decode_stack_noalloc(arr, x0, kind, y_last, y_layers, x_layers)
+        torch.cuda.synchronize()
+    else:
+        ws = torch.empty(ci.coreinfer_ffn_decode_stack_workspace_bytes(L, B, d, Kmax), dtype=torch.uint8, device="cuda")
+        ci.coreinfer_ffn_decode_stack(arr, x0, kind, y_last, y_layers, x_layers, ws)
+        ci.coreinfer_workspace_status(ws)
+    yl, xl = y_layers.cpu().numpy(), to_f32_np(x_layers)
+    assert np.isfinite(yl).all()
+    np.testing.assert_array_equal(xl[0], to_f32_np(x0))
+    np.testing.assert_allclose(y_last.cpu().numpy(), yl[L - 1], rtol=1e-4, atol=1e-5)
+    tol = 1e-5 if dtype == torch.float32 else 2 ** -7     # one rounding step of the layer-input type
+    for l in (range(L) if layers_to_check is None else layers_to_check):
+        up, gate, down, bup, bdown = (to_f32_np(t) for t in layers_gpu[l])
+        y_o = oracle.ffn(xl[l], kind, up, gate, down, bup, bdown)
+        assert_ffn_close(yl[l], y_o, dtype)
+        if l + 1 < L:
+            for b in range(B):
+                x_next = torch.from_numpy(oracle.glue(xl[l][b], yl[l][b])).to(dtype).float().numpy()
+                np.testing.assert_allclose(xl[l + 1][b], x_next.reshape(-1), rtol=tol, atol=tol)
+    return y_last, y_layers, x_layers

@@ -45,6 +45,9 @@ def test_argument_errors_are_reported_without_a_device(lib):
     assert b"NULL" in lib.coreinfer_last_error()
     assert lib.coreinfer_select_core(p, ci.F32, 4, 8, 8, 1.5, 0.2, p, null, p, 1024, null) == ci.ERR_INVALID_ARG
     assert lib.coreinfer_select_core(p, ci.BF16, 4, 8, 8, 0.4, 0.2, p, null, p, 1024, null) == ci.ERR_UNSUPPORTED
+    # a fraction inside (0, 1] that still rounds to an empty set
+    assert lib.coreinfer_select_core(p, ci.F32, 4, 8, 8, 0.4, 1e-9, p, null, p, 1024, null) == ci.ERR_INVALID_ARG
+    assert b"no neuron" in lib.coreinfer_last_error()
     assert lib.coreinfer_select_core(p, ci.F32, 4, 8, 8, 0.4, 0.2, p, null, p, 16, null) == ci.ERR_WORKSPACE
     # compaction: K out of range, gate given without its output
     assert lib.coreinfer_compact(p, null, p, null, ci.F32, 8, 16, p, 17, p, null, p, null, null) == ci.ERR_INVALID_ARG
@@ -53,7 +56,7 @@ def test_argument_errors_are_reported_without_a_device(lib):
     assert lib.coreinfer_ffn_decode(p, 9, ci.BF16, ci.FFN_RELU, 64, 4, p, null, p, null, null, p, p, 1024, null) == ci.ERR_UNSUPPORTED
     assert lib.coreinfer_ffn_decode(p, 1, ci.BF16, ci.FFN_RELU, 60, 4, p, null, p, null, null, p, p, 1024, null) == ci.ERR_INVALID_ARG
     assert lib.coreinfer_ffn_decode(p, 1, ci.BF16, ci.FFN_RELU_GATED, 64, 4, p, null, p, null, null, p, p, 1024, null) == ci.ERR_INVALID_ARG
-    # stack: batch 2 is not built, L out of range
+    # stack: batch beyond COREINFER_MAX_BATCH, L out of range
     layers = ci.binding.Layer * 1
     assert lib.coreinfer_ffn_decode_stack(layers(), 1, p, 9, ci.BF16, ci.FFN_RELU, 64, p, null, null, p, 1024, null) == ci.ERR_UNSUPPORTED
     assert lib.coreinfer_ffn_decode_stack(layers(), 0, p, 1, ci.BF16, ci.FFN_RELU, 64, p, null, null, p, 1024, null) == ci.ERR_INVALID_ARG

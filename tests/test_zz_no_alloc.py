@@ -1,13 +1,13 @@
 """The workspace-free stack entry point (for callers that cannot allocate device memory while
-decoding) must give what the workspace variant gives.  Collected last on purpose: a run that
-stops at the first failure has then already exercised every other test."""
+decoding) must give what the workspace variant gives, and what the oracle gives.  Collected last
+on purpose: a run that stops at the first failure has then already exercised every other test."""
 import numpy as np
 import pytest
 import torch
 
 import paper_2410_18311_b200 as ci
 from paper_2410_18311_b200 import workloads as wl
-from helpers import require_gpu, assert_ffn_close
+from helpers import require_gpu, assert_ffn_close, check_stack_teacher_forced
 
 pytestmark = pytest.mark.gpu
 
@@ -39,6 +39,10 @@ def test_noalloc_matches_workspace_variant_twice_in_a_row():
         assert_ffn_close(y.cpu().numpy(), y_ref.cpu().numpy(), torch.bfloat16)
         for l in range(L):
             assert_ffn_close(yl[l].cpu().numpy(), yl_ref[l].cpu().numpy(), torch.bfloat16)
+        # and against the oracle, layer by layer on the inputs the layers consumed (its private
+        # status word cannot be read back, so a wait that gave up would show here as a mismatch)
+        check_stack_teacher_forced([(u, g, dn, None, None) for (u, g, dn) in keep], x0, ci.FFN_RELU,
+                                   torch.bfloat16, noalloc=True)
     del keep
 
 
