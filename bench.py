@@ -27,10 +27,9 @@ METRIC = "core-sparse decode tokens/s at batch 1; achieved HBM GB/s vs B200 peak
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode_stack_kernel launch at the bench
-# workload: measured by ncu on a 4-layer launch of the same shapes (219.12 MB) and scaled by the
-# layer count, since every layer streams its own weights (profiles/decode_stack_kernel_opt6.7b.md).
-# Set to None whenever the kernel changes until the capture is repeated.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"opt6.7b": 219.12e6 / 4 * 32}
+# workload, from an ncu capture of a 4-layer launch of the same shapes scaled by the layer count
+# (every layer streams its own weights).  None whenever the kernel has changed since the capture.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"opt6.7b": None}
 
 
 def parse_args():
@@ -49,6 +48,9 @@ def parse_args():
                          "on random compacted weights (small enough for an ncu capture); prints a short JSON line")
     ap.add_argument("--tokens", type=int, default=2, help="decode launches per step in --decode-only mode")
     ap.add_argument("--batch", type=int, default=1, help="sequences per decode step in --decode-only mode (1..8)")
+    ap.add_argument("--stamps", action="store_true",
+                    help="with --decode-only: run the phase-timing build of the library (-DCOREINFER_STAMPS) and add "
+                         "the per-phase table of the last launch (median over CTAs and layers, microseconds)")
     ap.add_argument("--sequences", type=int, default=None,
                     help="also time the compacted stack for this many sequences sharing the core sets (2..8; "
                          "default: 8 for the gated Llama-shaped workload, which is specified at 1 and 8, else off)")
@@ -499,6 +501,8 @@ def run_decode_only(args, cfg):
     import paper_2410_18311_b200 as ci
     from paper_2410_18311_b200 import _build, workloads as wl
     _build.build()
+    if args.stamps:
+        ci.binding.use_library(_build.build(stamps=True))
     cfg = cfg.with_(L=args.decode_only)
     K = ci.coreinfer_count(cfg.beta, cfg.d_ff)
     layers = [wl.compacted_weights_random(cfg, l, K, device="cuda") for l in range(cfg.L)]
@@ -525,9 +529,46 @@ def run_decode_only(args, cfg):
     ci.coreinfer_workspace_status(ws)
     us = e0.elapsed_time(e1) * 1e3 / (args.steps * args.tokens)
     nbytes = cfg.L * cfg.n_mat * K * cfg.d_model * cfg.esize
-    print(json.dumps({"mode": "decode-only", "workload": cfg.name, "layers": cfg.L, "K": K, "batch": B,
-                      "us_per_launch": us, "us_per_layer": us / cfg.L, "bytes_per_launch": nbytes,
-                      "gbs": nbytes / us / 1e3, "sequence_tokens_per_s": B * 1e6 / us}), flush=True)
+    line = {"mode": "decode-only", "workload": cfg.name, "layers": cfg.L, "K": K, "batch": B,
+            "us_per_launch": us, "us_per_layer": us / cfg.L, "bytes_per_launch": nbytes,
+            "gbs": nbytes / us / 1e3, "sequence_tokens_per_s": B * 1e6 / us}
+    if args.stamps:
+        line["phases_us"] = phase_table(ci, lambda: ci.coreinfer_ffn_decode_stack(arr, xs[0], kind, ys[0], None, None, ws),
+                                        cfg.L, B)
+    print(json.dumps(line), flush=True)
+
+
+PHASES_B1 = [("up rows", 0, 1), ("h formed", 1, 2), ("down rows", 2, 3), ("partial assembled", 3, 4),
+             ("bulk reduction", 4, 5), ("release arrival", 5, 6), ("wait for all CTAs", 6, 7),
+             ("read-back", 7, 8), ("next input", 8, 9)]
+PHASES_BATCHED = [("up units", 0, 1), ("down units", 1, 3), ("flush of the partial", 3, 4),
+                  ("grid barrier", 4, 7), ("read-back of the sums", 7, 8), ("next input", 8, 9)]
+
+
+def phase_table(ci, launch, L, batch):
+    """One more launch with cycle stamps recorded (phase-timing build): per phase the median and
+    the mean over all CTAs and the layers 1 .. L-2, in microseconds at the SM clock sampled meanwhile."""
+    import torch
+    n_sm = torch.cuda.get_device_properties(0).multi_processor_count
+    stamps = torch.zeros((n_sm, L, ci.binding.STAMP_SLOTS), dtype=torch.int64, device="cuda")
+    ci.coreinfer_debug_stamps(stamps)
+    sampler = ClockSampler(0, period_s=0.01)
+    sampler.start()
+    for _ in range(20):
+        launch()
+    torch.cuda.synchronize()
+    mhz = sampler.stop()["sm_mhz"] or 1965
+    ci.coreinfer_debug_stamps(None)
+    st = stamps.cpu().double()
+    inner = st[:, 1:L - 1] if L > 2 else st
+    out = {"sm_mhz": mhz}
+    for name, a, b in (PHASES_B1 if batch == 1 else PHASES_BATCHED):
+        dt = (inner[:, :, b] - inner[:, :, a]).flatten() / mhz
+        out[name] = {"median": round(float(dt.median()), 3), "mean": round(float(dt.mean()), 3)}
+    if L > 2:
+        lay = (st[:, 2:, 0] - st[:, 1:-1, 0]).flatten() / mhz
+        out["layer"] = {"median": round(float(lay.median()), 3), "mean": round(float(lay.mean()), 3)}
+    return out
 
 
 def main():

@@ -13,8 +13,10 @@
  * Conventions for every entry point
  *   - "device" pointers are CUDA device memory of the current device; "host"
  *     pointers are ordinary host memory.  Every buffer is owned by the caller.
- *     The library allocates no device memory and keeps no state between calls
- *     except a thread-local error string.
+ *     The library allocates no device memory.  Between calls it keeps a
+ *     thread-local error string, per-device properties it looked up once, and
+ *     the fixed scratch array of coreinfer_ffn_decode_stack_noalloc (whose
+ *     contents carry no meaning from one call to the next).
  *   - Matrices are row-major and dense.  Device pointers must be 16-byte
  *     aligned; d_model * sizeof(element) must be a multiple of 16.
  *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = default stream).
@@ -225,6 +227,21 @@ coreinfer_status coreinfer_ffn_decode_stack_noalloc(const coreinfer_layer* layer
  * if a bounded device-side wait gave up (outputs of that call are then
  * undefined).  Returns COREINFER_ERR_CUDA if the synchronisation or copy fails. */
 coreinfer_status coreinfer_workspace_status(const void* workspace, void* cuda_stream);
+
+/* Phase timing of the persistent decode kernels (a profiling aid; the paper has no counterpart).
+ * Only a library built with -DCOREINFER_STAMPS records anything; the normal build returns
+ * COREINFER_ERR_UNSUPPORTED.  After this call, every coreinfer_ffn_decode_stack launch made
+ * from the calling thread stores the SM cycle counter (clock64) at fixed points of each layer
+ * into `stamps`: device, [CTAs = SM count][L][COREINFER_STAMP_SLOTS] 64-bit words, as long as
+ * `bytes` covers that; launches with more layers than fit record nothing.  Batch-1 slots:
+ * 0 layer start, 1 up rows consumed, 2 h formed, 3 down rows consumed, 4 the CTA's partial y
+ * assembled, 5 its bulk reduction complete, 6 arrival at the grid barrier issued, 7 all CTAs
+ * arrived, 8 sum read back, 9 next input formed.  For 2..8 sequences: 0 layer start, 1 up units
+ * done, 3 down units done, 4 partial flushed, 7 all CTAs arrived, 8 sums read back, 9 next input
+ * formed.  Slots not listed stay untouched.  NULL switches recording off.  The buffer is the
+ * caller's and must outlive the launches. */
+#define COREINFER_STAMP_SLOTS 16
+coreinfer_status coreinfer_debug_stamps(void* stamps, size_t bytes);
 
 /* ------------------------------------------------------------------ (4) --
  * Dense FFN on the uncompacted weights: the pre-fill pass whose intermediate

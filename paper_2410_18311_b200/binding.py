@@ -28,8 +28,10 @@ SYMBOLS = (
     "coreinfer_ffn_decode_stack_workspace_bytes", "coreinfer_ffn_decode_stack",
     "coreinfer_ffn_decode_stack_noalloc",
     "coreinfer_workspace_status",
+    "coreinfer_debug_stamps",
     "coreinfer_ffn_dense_ref",
 )
+STAMP_SLOTS = 16
 
 
 class CoreInferError(RuntimeError):
@@ -46,10 +48,17 @@ class Layer(ctypes.Structure):
 
 
 _lib = None
+_lib_path = None
 
 
 def library_path() -> str:
-    return _build.LIB_PATH
+    return _lib_path or _build.LIB_PATH
+
+
+def use_library(path: str) -> None:
+    """Make every later call go to another build of the library (the phase-timing variant)."""
+    global _lib, _lib_path
+    _lib, _lib_path = None, path
 
 
 def load() -> ctypes.CDLL:
@@ -88,6 +97,8 @@ def load() -> ctypes.CDLL:
                                                        ctypes.c_int, i32, vp, vp, vp, vp]
     lib.coreinfer_workspace_status.restype = ctypes.c_int
     lib.coreinfer_workspace_status.argtypes = [vp, vp]
+    lib.coreinfer_debug_stamps.restype = ctypes.c_int
+    lib.coreinfer_debug_stamps.argtypes = [vp, sz]
     lib.coreinfer_ffn_dense_ref.restype = ctypes.c_int
     lib.coreinfer_ffn_dense_ref.argtypes = [vp, i32, ctypes.c_int, ctypes.c_int, i32, i32, vp, vp, vp, vp, vp,
                                             vp, vp, vp]
@@ -205,6 +216,12 @@ def coreinfer_ffn_decode_stack_noalloc(layers, x0, kind, y_last, y_layers, x_lay
 def coreinfer_workspace_status(workspace, stream=None) -> None:
     """Synchronises the stream; raises CoreInferError(ERR_TIMEOUT) if a device-side wait gave up."""
     _check(load().coreinfer_workspace_status(_p(workspace), _stream(stream)))
+
+
+def coreinfer_debug_stamps(stamps) -> None:
+    """stamps: CUDA int64 tensor [CTAs, L, STAMP_SLOTS] that later stack launches fill with cycle
+    counts, or None to stop recording.  Raises ERR_UNSUPPORTED unless the phase-timing build is loaded."""
+    _check(load().coreinfer_debug_stamps(_p(stamps), 0 if stamps is None else stamps.numel() * stamps.element_size()))
 
 
 def coreinfer_ffn_dense_ref(x, kind, w_up, w_gate, w_down, b_up, b_down, h_out, y_out, stream=None):

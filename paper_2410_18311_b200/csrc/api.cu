@@ -17,6 +17,14 @@ void set_error(const char* fmt, ...)
     va_end(ap);
 }
 
+static thread_local unsigned long long* g_stamps = nullptr;
+static thread_local size_t g_stamps_bytes = 0;
+
+unsigned long long* stamps_buffer(size_t need_bytes)
+{
+    return (g_stamps && g_stamps_bytes >= need_bytes) ? g_stamps : nullptr;
+}
+
 coreinfer_status device_info(DeviceInfo* out)
 {
     static thread_local DeviceInfo cache[64];
@@ -58,6 +66,21 @@ int32_t coreinfer_count(double frac, int32_t n)
 }
 
 const char* coreinfer_last_error(void) { return coreinfer::g_error; }
+
+coreinfer_status coreinfer_debug_stamps(void* stamps, size_t bytes)
+{
+#ifdef COREINFER_STAMPS
+    if (stamps && (reinterpret_cast<uintptr_t>(stamps) & 7u))
+        CI_FAIL(COREINFER_ERR_INVALID_ARG, "stamps must be 8-byte aligned");
+    coreinfer::g_stamps = (unsigned long long*)stamps;
+    coreinfer::g_stamps_bytes = stamps ? bytes : 0;
+    return COREINFER_OK;
+#else
+    (void)stamps;
+    (void)bytes;
+    CI_FAIL(COREINFER_ERR_UNSUPPORTED, "this library was built without COREINFER_STAMPS");
+#endif
+}
 
 coreinfer_status coreinfer_workspace_status(const void* workspace, void* cuda_stream)
 {

@@ -41,6 +41,21 @@ struct DeviceInfo {
 };
 coreinfer_status device_info(DeviceInfo* out);
 
+// Optional phase timing.  Built with -DCOREINFER_STAMPS, the persistent decode kernels store the
+// SM cycle counter at fixed points of every layer into the buffer registered with
+// coreinfer_debug_stamps(): [CTA][layer][kStampSlots] 64-bit words.  In the normal build
+// the macro is empty and the registration call reports UNSUPPORTED.
+constexpr int kStampSlots = 16;
+unsigned long long* stamps_buffer(size_t need_bytes);   // NULL unless a large enough buffer is registered
+#ifdef COREINFER_STAMPS
+#define CI_STAMP(buf, base, id)                                  \
+    do {                                                         \
+        if (buf) (buf)[(base) + (id)] = (unsigned long long)clock64(); \
+    } while (0)
+#else
+#define CI_STAMP(buf, base, id) do { } while (0)
+#endif
+
 // --------------------------------------------------------------- device -----
 // Status word values written by kernels (first word of a decode workspace).
 enum : unsigned { kStatusOk = 0u, kStatusTimeout = 5u };
@@ -99,7 +114,7 @@ __device__ __forceinline__ bool mbar_try_wait_parked(uint32_t bar, uint32_t pari
 }
 
 // 1-D bulk copy global -> shared of this CTA, completion counted on an mbarrier.
-// dst, src 16-byte aligned; bytes a multiple of 16.  No multicast.
+// dst, src 16-byte aligned; bytes a multiple of 16.  The copy targets this CTA alone.
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
 {
     asm volatile(

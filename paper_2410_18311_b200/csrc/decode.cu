@@ -3,39 +3,40 @@
 // One persistent kernel, one CTA per SM.  Per layer a CTA owns a contiguous slab of the K core
 // neurons and streams that slab's rows exactly once: first the up (and gate) rows to form h for
 // its neurons, then the matching rows of the transposed down matrix to form its partial y.
-// Rows arrive through a ring of shared-memory slots filled by 1-D bulk copies (a producer warp,
-// one full/empty mbarrier pair per slot).  The weights of a layer do not depend on its input,
-// so the producer runs ahead across layer boundaries and HBM stays busy while the CTAs exchange
-// partial outputs.
+// Rows arrive in batches of BATCH rows through a ring of shared-memory batch slots filled by 1-D
+// bulk copies (a producer warp; one full/empty mbarrier pair per batch slot, all rows of a batch
+// complete on the same barrier).  The weights of a layer do not depend on its input, so the
+// producer runs ahead across layer boundaries.
 //
-// Consumers own columns: thread t of a group holds the x values of its 16-byte vectors
-// t, t + 256, ... in registers for the whole layer and its partial y likewise.  They take ring
-// items in batches: wait for the batch, pull every vector of all its rows into registers with
-// no branch in between (so the loads overlap), free the slots at once, and only then do the
-// arithmetic; slots are held for a few hundred cycles whatever the arithmetic costs.  For rows
-// of at most 8 KB two such groups take alternate batches, so that one group's shared-memory
-// reads overlap the other's arithmetic; wider rows use one group.
+// Consumers own columns: thread t holds the x values of its 16-byte vectors t, t + NC, ... in
+// registers for the whole layer and its partial y likewise.  They walk the stream of batches with
+// two register buffers: the rows of the next batch are requested from shared memory (one barrier
+// test, BATCH * VPT 16-byte loads, the slot freed at once) before the arithmetic of the current
+// batch starts, so that barrier and shared-memory latencies are hidden behind the arithmetic; the
+// per-row costs of a warp are one sixteen-byte load per vector and its multiply-adds.
 //
 // Exchange per layer: the CTA's partial y (d_model fp32) is assembled in shared memory and added
 // into a global vector with one bulk reduction; one thread waits for it, arrives at a grid
 // barrier (release), polls for everybody else's arrival (acquire) and brings the sum back with
-// one bulk copy, on whose barrier the other consumers sleep; every group then forms the next
-// layer's input redundantly in registers.  Every wait (slot barriers, grid barrier, read-back)
-// is bounded: when one gives up, the CTA marks the workspace status word, stops waiting
-// everywhere, runs the rest of its schedule without synchronising on data, drains its own
-// copies in flight and returns.
+// one bulk copy, on whose barrier the other consumers sleep; every thread then forms its columns
+// of the next layer's input.  While the exchange is on, the producer requests only a limited
+// number of rows: a first part before the exchange (landed by then), a second part once this
+// CTA's arrival is out (a fence waits for the SM's bulk copies in flight, so none is issued
+// before), paced.  Every wait (slot barriers, grid barrier, read-back) is bounded: when one gives
+// up, the CTA marks the workspace status word, stops waiting everywhere, runs the rest of its
+// schedule without synchronising on data, drains its own copies in flight and returns.
 #include "common.cuh"
 
 #include <stdlib.h>
 
 namespace coreinfer {
 
-constexpr int kMaxSlots = 64;
-constexpr int kGroupThreads = 256;                     // consumer threads per group
-constexpr int kGroupWarps = kGroupThreads / 32;
+constexpr int kMaxBatchSlots = 64;
+constexpr int kMaxConsumers = 512;                     // consumer threads per CTA (16 warps) + one producer warp
+constexpr int kMaxWarps = kMaxConsumers / 32;
+constexpr int kMaxVpt = 3;                             // 16-byte vectors of a row per consumer thread
 constexpr int kCtrlBytes = 256;                        // status word, barrier counter, padding
-constexpr int kYCopies = 1;                            // copies of a reduction target (more spread same-address adds, but cost more to read back)
-constexpr int kYBuffers = 3;                           // rotating targets: in use, being read, being cleared
+constexpr int kYBuffers = 3;                           // rotating reduction targets: in use, being read, being cleared
 constexpr int kSplitRotate = 41;                       // per-layer rotation of the slab split
 constexpr long long kWaitCycles = 3000000000LL;        // bound of every device-side wait (~1.5 s)
 
@@ -50,16 +51,20 @@ struct LayerDev {
 };
 
 struct DecodeParams {
-    int L, d, nv, row_bytes, slot_bytes, n_slots, rmax;
-    int runahead;       // ring items of the next layer the producer may request before this layer's exchange is over
+    int L, d, nv, row_bytes, slot_bytes, n_bslots, rmax;
+    int nc;             // consumer threads (a multiple of 32); the producer warp follows them
+    int runahead;       // batches of the next layer requested before this layer's exchange is over
+    int trickle;        // further batches, requested one by one once this CTA's arrival at the grid barrier is out
+    int trickle_gap;    // cycles between two such requests
     float inv_d;        // 1 / d_model
     int ysum_ofs;       // shared-memory offset of the buffer holding the CTA's partial y
     const void* x0;
     float* y_last;
     float* y_layers;
     void* x_layers;
-    float* ybuf;        // [kYBuffers][kYCopies][d]: reduction targets, buffer l % 3 serves layer l
+    float* ybuf;        // [kYBuffers][d]: reduction targets, buffer l % 3 serves layer l
     unsigned* ctrl;     // [0] status word, [1] grid-barrier arrival counter
+    unsigned long long* stamps;   // [CTA][layer][kStampSlots] cycle counts, or NULL (COREINFER_STAMPS builds)
     LayerDev layers[COREINFER_MAX_LAYERS];
 };
 
@@ -73,11 +78,10 @@ __host__ __device__ __forceinline__ void slab_of(int cta, int G, int layer, int 
     *k1 = (int)((vc + 1u) * (unsigned)K / g);
 }
 
-// items per consumer batch for one group (register budget: 4 * items * vectors per thread)
-__host__ __device__ constexpr int batch_for(int groups, int vpt)
-{
-    return groups == 2 ? 4 : (vpt <= 2 ? 8 : (vpt <= 4 ? 4 : 2));
-}
+// rows per batch (register budget: two buffers of 4 * rows * vectors per thread)
+__host__ __device__ constexpr int batch_for(int vpt) { return vpt <= 1 ? 4 : 2; }
+// consumer threads at most: with three vectors per thread 14 warps, which leaves 128 registers a thread
+__host__ __device__ constexpr int max_consumers(int vpt) { return vpt <= 2 ? kMaxConsumers : 448; }
 
 // ------------------------------------------------------------ element types --
 template <typename T> struct Elem;
@@ -161,14 +165,13 @@ __device__ __forceinline__ bool wait_slot(uint32_t bar, uint32_t parity, volatil
     }
 }
 
-// One thread per CTA calls this, after it has seen the CTA's work complete.  The arrival
-// counter is zeroed by the host before the launch; barrier number b (0-based) completes when it
-// reaches (b + 1) * G.  The arrival is a release at GPU scope (what this thread has observed,
-// the completed bulk reduction and the CTA's earlier plain writes included, becomes visible
-// before it), the poll an acquire.
-__device__ __forceinline__ void grid_arrive_and_wait(unsigned* ctrl, unsigned target, volatile int* abort_flag)
+// Grid barrier: one thread per CTA, after it has seen the CTA's work complete, arrives with
+// red_release_add(&ctrl[1], 1) and then calls this.  The arrival counter is zeroed by the host
+// before the launch; barrier number b (0-based) completes when it reaches (b + 1) * G.  The
+// arrival is a release at GPU scope (what this thread has observed, the completed bulk reduction
+// and the CTA's earlier plain writes included, becomes visible before it), the poll an acquire.
+__device__ __forceinline__ void grid_wait(unsigned* ctrl, unsigned target, volatile int* abort_flag)
 {
-    red_release_add(&ctrl[1], 1u);
     const long long t0 = clock64();
     unsigned it = 0;
     for (;;) {
@@ -214,130 +217,179 @@ __device__ __forceinline__ float warp_reduce8(const float (&v)[8], int lane)
     return c;
 }
 
+// 4 values per lane -> 4 warp totals, one per group of 8 lanes (5 shuffles).
+// On return lane l holds the total of value ((l>>4)&1)*2 + ((l>>3)&1).
+__device__ __forceinline__ float warp_reduce4(const float (&v)[4], int lane)
+{
+    float a[2];
+    const bool hi16 = lane & 16;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        float send = hi16 ? v[i] : v[i + 2];
+        float keep = hi16 ? v[i + 2] : v[i];
+        a[i] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+    }
+    const bool hi8 = lane & 8;
+    float send = hi8 ? a[0] : a[1];
+    float keep = hi8 ? a[1] : a[0];
+    float c = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+    c += __shfl_xor_sync(0xffffffffu, c, 4);
+    c += __shfl_xor_sync(0xffffffffu, c, 2);
+    c += __shfl_xor_sync(0xffffffffu, c, 1);
+    return c;
+}
+
+__device__ __forceinline__ float warp_reduce_n(const float (&v)[8], int lane) { return warp_reduce8(v, lane); }
+__device__ __forceinline__ float warp_reduce_n(const float (&v)[4], int lane) { return warp_reduce4(v, lane); }
+
 // ------------------------------------------------------------------- kernel --
 // Ring stream order of one CTA and one layer (producer and consumers walk it in lock step): for
 // each slab row k0 .. k1-1 its up row, then (gated) its gate row; after those, the down rows
-// k0 .. k1-1.  Within each of the two phases the items are cut into batches of BATCH.  With two
-// consumer groups every batch takes BATCH ring slots, the last batch of a phase being filled up
-// with empty items (no copy: the producer completes their barrier by a plain arrival), and the
-// batches of the whole launch are dealt out in turn: batch number g of the launch belongs to
-// group g % NG and starts at ring position (g * BATCH) % slots.  The ring holds a multiple of
-// NG * BATCH slots, so a slot is read by the same group in every pass of the ring: a group that
-// tests a slot's barrier has itself consumed the slot's previous fill, and can therefore never
-// mistake the parity of a fill that is still in flight for that of the one it wants.
-template <typename T, int NG, int VPT, bool GATED>
-__global__ void __launch_bounds__(NG * kGroupThreads + 32, 1)
+// k0 .. k1-1.  Each of the two phases is cut into batches of BATCH rows (the last one of a phase
+// may hold fewer); every batch takes one batch slot of the ring, whatever it holds.
+template <typename T, int VPT, bool GATED>
+__global__ void __launch_bounds__(max_consumers(VPT) + 32, 1)
 decode_stack_kernel(const __grid_constant__ DecodeParams p)
 {
     using E = Elem<T>;
     constexpr int PAIRS = E::kPairs;
     constexpr int EPV = PAIRS * 2;                   // elements per 16-byte vector
     constexpr int NMAT = GATED ? 2 : 1;
-    constexpr int NC = NG * kGroupThreads;           // consumer threads
-    constexpr int BATCH = batch_for(NG, VPT);        // ring items per batch
-    constexpr int PADB = NG > 1 ? BATCH : 1;         // a phase takes a multiple of PADB ring slots
-    constexpr int FLUSH = 16 / BATCH;                // own up batches per cross-lane reduction (16 row sums)
+    constexpr int BATCH = batch_for(VPT);            // rows per batch
+    constexpr int WIN = 2 * BATCH;                   // row sums per cross-lane reduction: one turn of the two register buffers
 
     extern __shared__ __align__(128) uint8_t smem[];
+    const int NB = p.n_bslots;
+    const int NC = p.nc;
+    const int nwarps = NC >> 5;
+    const uint32_t bslot_bytes = (uint32_t)BATCH * (uint32_t)p.slot_bytes;
     uint8_t* ring = smem;
-    uint64_t* full_bar = reinterpret_cast<uint64_t*>(ring + (size_t)p.n_slots * p.slot_bytes);
-    uint64_t* empty_bar = full_bar + kMaxSlots;
-    uint64_t* y_bar = empty_bar + kMaxSlots;                        // completion of the read-back copy (+ 8 bytes padding)
-    float* red = reinterpret_cast<float*>(y_bar + 2);               // [NMAT][kGroupWarps][rmax]
-    float* h_s = red + NMAT * kGroupWarps * p.rmax;                 // [rmax]
-    float* ss_red = h_s + p.rmax;                                   // [NG][kGroupWarps]
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(ss_red + NG * kGroupWarps);
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(ring + (size_t)NB * bslot_bytes);
+    uint64_t* empty_bar = full_bar + kMaxBatchSlots;
+    uint64_t* y_bar = empty_bar + kMaxBatchSlots;                   // completion of the read-back copy (+ 8 bytes padding)
+    float* red = reinterpret_cast<float*>(y_bar + 2);               // [NMAT][nwarps][rmax]
+    float* h_s = red + NMAT * nwarps * p.rmax;                      // [rmax]
+    float* ss_red = h_s + p.rmax;                                   // [kMaxWarps]
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(ss_red + kMaxWarps);
     volatile int* layers_done = abort_flag + 1;                     // layers whose exchange this CTA has completed
-    float* ysum = reinterpret_cast<float*>(smem + p.ysum_ofs);      // [VPT * 256 * EPV]: the CTA's partial y
+    volatile int* arrived = abort_flag + 2;                         // layers for which this CTA's grid-barrier arrival is out
+    float* ysum = reinterpret_cast<float*>(smem + p.ysum_ofs);      // [d]: the CTA's partial y, then the sum
 
     const int tid = threadIdx.x;
     const int G = gridDim.x;
     const int cta = blockIdx.x;
-    const int NS = p.n_slots;
 
     if (tid == 0) {
-        for (int s = 0; s < NS; ++s) {
+        for (int s = 0; s < NB; ++s) {
             mbar_init(smem_u32(&full_bar[s]), 1);
-            mbar_init(smem_u32(&empty_bar[s]), kGroupWarps);     // the warps of the group that reads the slot
+            mbar_init(smem_u32(&empty_bar[s]), (uint32_t)nwarps);   // one arrival per consumer warp
         }
         mbar_init(smem_u32(y_bar), 1);
         *abort_flag = 0;
         *layers_done = 0;
+        *arrived = 0;
         mbar_fence_init();
     }
     __syncthreads();
 
     // ======================================================== producer warp ==
-    // Up to eight lanes issue copies: one round fills up to min(8, ring slots) consecutive ring
-    // items, lane j taking item j of the round (its own slot, its own wait on that slot's
-    // "empty" barrier), so the latency of one issue is not the issue rate.
+    // Eight lanes issue copies: one round fills up to 8 / BATCH consecutive batch slots, lane j
+    // taking row j % BATCH of batch j / BATCH of the round.  Every lane waits for its batch slot to
+    // be free; the lane of the batch's first row announces the bytes of the whole batch.
     if (tid >= NC) {
         const int lane = tid - NC;
-        const int round_max = NS < 8 ? NS : 8;
-        int slot0 = 0;                // ring position of the round's first item
-        uint32_t phase0 = 0;          // parity of the ring pass that position belongs to
-        long long issued = 0;
+        constexpr int RB = 8 / BATCH;
+        const int round_max = NB < RB ? NB : RB;
+        int bs0 = 0;                  // batch slot of the round's first batch
+        uint32_t phase0 = 0;          // parity of the ring pass that slot belongs to
+        long long issued = 0;         // batches
         for (int l = 0; l < p.L; ++l) {
             const LayerDev& ly = p.layers[l];
             int k0, k1;
             slab_of(cta, G, l, ly.K, &k0, &k1);
             const int n = k1 - k0;
-            const int n_up = n * NMAT;            // items of the up (+ gate) phase
-            const int p_up = (n_up + PADB - 1) / PADB * PADB;          // ring slots of that phase
-            const int total = p_up + (n + PADB - 1) / PADB * PADB;     // + those of the down rows
-            for (int q0 = 0, cnt = 0; q0 < total; q0 += cnt) {
+            const int n_up = n * NMAT;                               // rows of the up (+ gate) phase
+            const int nbu = (n_up + BATCH - 1) / BATCH;              // its batches
+            const int nbt = nbu + (n + BATCH - 1) / BATCH;           // + those of the down rows
+            long long t_next = 0;                                    // earliest time of the next paced request
+            for (int b0 = 0, cnt = 0; b0 < nbt; b0 += cnt) {
                 if (*abort_flag) break;
-                cnt = min(round_max, total - q0);
-                // Every weight request in flight delays the few small messages of the previous
-                // layer's exchange (adds, arrival, poll, read-back), which queue behind it.  So
-                // only a limited number of this layer's rows is requested before that exchange is
-                // over: a round is cut at the limit, and beyond it the producer waits.
-                if (l > 0 && q0 + cnt > p.runahead && *layers_done < l) {
-                    if (q0 < p.runahead) {
-                        cnt = p.runahead - q0;
+                cnt = min(round_max, nbt - b0);
+                // Requests in flight delay the few small messages of the previous layer's exchange,
+                // and its fence waits for this SM's copies in flight.  So while that exchange is on,
+                // only `runahead` batches of this layer are requested at once (they have landed
+                // when the exchange starts); `trickle` more follow one at a time, `trickle_gap`
+                // cycles apart, after this CTA's arrival at the grid barrier is out; the rest wait
+                // for the end of the exchange.  Lane 0 decides for the warp.
+                int limited = 0;
+                if (l > 0 && b0 + cnt > p.runahead) {
+                    limited = *layers_done < l;
+                    limited = __shfl_sync(0xffffffffu, limited, 0);
+                }
+                if (limited) {
+                    if (b0 < p.runahead) {
+                        cnt = p.runahead - b0;
                     } else {
-                        const long long t0 = clock64();
-                        while (*layers_done < l && !*abort_flag) {
-                            __nanosleep(64);
-                            if (clock64() - t0 > kWaitCycles) { *abort_flag = 1; atomicMax(p.ctrl, (unsigned)kStatusTimeout); }
+                        int go = 0;                                  // 1: one paced batch, 2: the exchange is over
+                        if (lane == 0) {
+                            const long long t0 = clock64();
+                            for (;;) {
+                                if (*layers_done >= l || *abort_flag) { go = 2; break; }
+                                const long long now = clock64();
+                                if (b0 < p.runahead + p.trickle && *arrived >= l && now >= t_next) {
+                                    t_next = now + p.trickle_gap;
+                                    go = 1;
+                                    break;
+                                }
+                                __nanosleep(32);
+                                if (now - t0 > kWaitCycles) { *abort_flag = 1; atomicMax(p.ctrl, (unsigned)kStatusTimeout); }
+                            }
                         }
+                        go = __shfl_sync(0xffffffffu, go, 0);
+                        if (go == 1) cnt = 1;
                     }
                 }
-                if (lane < cnt) {
-                    const int q = q0 + lane;
-                    const uint8_t* src = nullptr;         // stays NULL for an empty item
-                    if (q < n_up) {
-                        const int row = k0 + q / NMAT;
-                        src = ((GATED && (q % NMAT)) ? ly.gate : ly.up) + (size_t)row * p.row_bytes;
-                    } else if (q >= p_up && q - p_up < n) {
-                        src = ly.down + (size_t)(k0 + q - p_up) * p.row_bytes;
+                if (lane < cnt * BATCH) {
+                    const int bi = lane / BATCH, r = lane % BATCH;
+                    const int b = b0 + bi;
+                    const uint8_t* src = nullptr;                    // stays NULL for a row the batch does not hold
+                    int nreal;
+                    if (b < nbu) {
+                        const int q = b * BATCH + r;
+                        nreal = min(BATCH, n_up - b * BATCH);
+                        if (q < n_up)
+                            src = ((GATED && (q % NMAT)) ? ly.gate : ly.up) + (size_t)(k0 + q / NMAT) * p.row_bytes;
+                    } else {
+                        const int q = (b - nbu) * BATCH + r;
+                        nreal = min(BATCH, n - (b - nbu) * BATCH);
+                        if (q < n) src = ly.down + (size_t)(k0 + q) * p.row_bytes;
                     }
-                    int sl = slot0 + lane;
+                    int bs = bs0 + bi;
                     uint32_t ph = phase0;
-                    if (sl >= NS) { sl -= NS; ph ^= 1u; }
-                    if (wait_slot(smem_u32(&empty_bar[sl]), ph ^ 1u, abort_flag, p.ctrl)) {
-                        const uint32_t fb = smem_u32(&full_bar[sl]);
-                        if (src) {
-                            mbar_arrive_expect_tx(fb, (uint32_t)p.row_bytes);
-                            bulk_g2s(smem_u32(ring + (size_t)sl * p.slot_bytes), src, (uint32_t)p.row_bytes, fb);
-                        } else {
-                            mbar_arrive(fb);
-                        }
+                    if (bs >= NB) { bs -= NB; ph ^= 1u; }
+                    if (wait_slot(smem_u32(&empty_bar[bs]), ph ^ 1u, abort_flag, p.ctrl)) {
+                        const uint32_t fb = smem_u32(&full_bar[bs]);
+                        // (a copy of another lane may complete before this announcement: the barrier's
+                        // pending arrival keeps the phase open until the announcement is made)
+                        if (r == 0) mbar_arrive_expect_tx(fb, (uint32_t)nreal * (uint32_t)p.row_bytes);
+                        if (src)
+                            bulk_g2s(smem_u32(ring + (size_t)bs * bslot_bytes + (size_t)r * p.slot_bytes), src,
+                                     (uint32_t)p.row_bytes, fb);
                     }
                 }
                 __syncwarp();
-                slot0 += cnt;
-                if (slot0 >= NS) { slot0 -= NS; phase0 ^= 1u; }
+                bs0 += cnt;
+                if (bs0 >= NB) { bs0 -= NB; phase0 ^= 1u; }
                 issued += cnt;
             }
         }
         // Do not leave while a copy into this CTA's shared memory is in flight: wait (bounded)
-        // for the last copy issued into every slot.  (After an abort a counted item may not have
+        // for the last fill of every batch slot.  (After an abort a counted batch may not have
         // been issued; its wait then runs into the bound, which only delays the return.)
-        for (int sl = lane; sl < NS; sl += 32) {
-            const long long uses = issued / NS + (sl < (int)(issued % NS) ? 1 : 0);
+        for (int bs = lane; bs < NB; bs += 32) {
+            const long long uses = issued / NB + (bs < (int)(issued % NB) ? 1 : 0);
             if (uses == 0) continue;
-            const uint32_t fb = smem_u32(&full_bar[sl]);
+            const uint32_t fb = smem_u32(&full_bar[bs]);
             const uint32_t ph = (uint32_t)((uses - 1) & 1);
             const long long t0 = clock64();
             while (!mbar_try_wait(fb, ph))
@@ -347,190 +399,124 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
     }
 
     // ============================================================ consumers ==
-    const int grp = tid / kGroupThreads;          // consumer group of this thread
-    const int gt = tid % kGroupThreads;           // thread within the group
     const int lane = tid & 31;
-    const int gw = gt >> 5;                       // warp within the group
+    const int warp = tid >> 5;
     const int nv = p.nv;
     const int d = p.d;
 
-    // this thread's columns: 16-byte vectors gt, gt + 256, ...  vofs[] is clamped so that loads
+    // this thread's columns: 16-byte vectors tid, tid + NC, ...  vofs[] is clamped so that loads
     // never need a branch (threads beyond the row read vector 0 against a zero x).
     uint4 xq[VPT];                // x in the weight type, as loaded
     int vofs[VPT];
 #pragma unroll
     for (int i = 0; i < VPT; ++i) {
-        const int v = gt + i * kGroupThreads;
+        const int v = tid + i * NC;
         vofs[i] = (v < nv ? v : 0) * 16;
         uint4 q = make_uint4(0, 0, 0, 0);
         if (v < nv) q = reinterpret_cast<const uint4*>(p.x0)[v];
         xq[i] = q;
-        if (p.x_layers && cta == 0 && grp == 0 && v < nv) reinterpret_cast<uint4*>(p.x_layers)[v] = q;
+        if (p.x_layers && cta == 0 && v < nv) reinterpret_cast<uint4*>(p.x_layers)[v] = q;
     }
 
-    int slot = 0;                 // ring position of the next item of the stream
+    int bslot = 0;                // batch slot of the next batch of the stream
     uint32_t phase = 0;
-    int gbatch = 0;               // two groups: number, within the launch, of the current phase's first batch
-    auto skip_n = [&](int n) {    // ring slots that belong to the other group
-        slot += n;
-        if (slot >= NS) { slot -= NS; phase ^= 1u; }
-    };
-    // wait for the next n items, pull them into registers (q[j][i] = vector i of item j), free them
-    auto fetch = [&](uint4 (&q)[BATCH][VPT], int n) {
-        const int held = NG > 1 ? BATCH : n;      // ring slots of this batch (two groups: empty items included)
-        {
-            // test all barriers of the batch back to back (the tests overlap); only if one is
-            // not complete yet fall back to the bounded waits, one by one
-            bool ready = true;
+    const uint32_t ring_u32 = smem_u32(ring);
+    // wait for the next batch, request its rows from shared memory (q[j][i] = vector i of row j),
+    // free the slot.  The loads of one warp are performed in order with its arrival that follows.
+    auto fetch = [&](uint4 (&q)[BATCH][VPT]) {
+        const uint32_t fb = smem_u32(&full_bar[bslot]);
+        if (!mbar_try_wait(fb, phase)) wait_slot(fb, phase, abort_flag, p.ctrl);
+        const uint32_t base = ring_u32 + (uint32_t)bslot * bslot_bytes;
 #pragma unroll
-            for (int j = 0; j < BATCH; ++j) {
-                int sl = slot + (j < held ? j : 0);
-                uint32_t ph = phase;
-                if (sl >= NS) { sl -= NS; ph ^= 1u; }
-                ready &= mbar_try_wait(smem_u32(&full_bar[sl]), ph);
-            }
-            if (!ready) {
-                int sl = slot;
-                uint32_t ph = phase;
-                for (int j = 0; j < held; ++j) {
-                    wait_slot(smem_u32(&full_bar[sl]), ph, abort_flag, p.ctrl);
-                    if (++sl == NS) { sl = 0; ph ^= 1u; }
-                }
-            }
-        }
-        if (n == BATCH) {
+        for (int j = 0; j < BATCH; ++j)
 #pragma unroll
-            for (int j = 0; j < BATCH; ++j) {
-                int sl = slot + j;
-                if (sl >= NS) sl -= NS;
-                const uint8_t* row = ring + (size_t)sl * p.slot_bytes;
-#pragma unroll
-                for (int i = 0; i < VPT; ++i) q[j][i] = *reinterpret_cast<const uint4*>(row + vofs[i]);
-            }
-        } else {
-#pragma unroll
-            for (int j = 0; j < BATCH; ++j) {
-                int sl = slot + (j < n ? j : 0);
-                if (sl >= NS) sl -= NS;
-                const uint8_t* row = ring + (size_t)sl * p.slot_bytes;
-#pragma unroll
-                for (int i = 0; i < VPT; ++i) {
-                    q[j][i] = *reinterpret_cast<const uint4*>(row + vofs[i]);
-                    if (j >= n) q[j][i] = make_uint4(0, 0, 0, 0);
-                }
-            }
-        }
+            for (int i = 0; i < VPT; ++i)
+                asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                             : "=r"(q[j][i].x), "=r"(q[j][i].y), "=r"(q[j][i].z), "=r"(q[j][i].w)
+                             : "r"(base + (uint32_t)j * (uint32_t)p.slot_bytes + (uint32_t)vofs[i]));
         __syncwarp();
-        if (lane < held && !*abort_flag) {
-            int sl = slot + lane;
-            if (sl >= NS) sl -= NS;
-            mbar_arrive(smem_u32(&empty_bar[sl]));
-        }
-        skip_n(held);
+        if (lane == 0) mbar_arrive(smem_u32(&empty_bar[bslot]));
+        if (++bslot == NB) { bslot = 0; phase ^= 1u; }
     };
 
+    unsigned long long* const stamps = tid == 0 ? p.stamps : nullptr;   // thread 0 runs the exchange
     for (int l = 0; l < p.L; ++l) {
         const LayerDev& ly = p.layers[l];
         int k0, k1;
         slab_of(cta, G, l, ly.K, &k0, &k1);
         const int nrows = k1 - k0;
         const int n_up = nrows * NMAT;
+        const int nbu = (n_up + BATCH - 1) / BATCH;
+        const int nbt = nbu + (nrows + BATCH - 1) / BATCH;
+        const size_t sb = ((size_t)cta * p.L + l) * kStampSlots;
+        (void)sb;
+        CI_STAMP(stamps, sb, 0);
 
-        // ------------------------------------------------ up (+ gate) phase --
-        {
-            const int nb = (n_up + BATCH - 1) / BATCH;
-            float part[16];
-#pragma unroll
-            for (int j = 0; j < 16; ++j) part[j] = 0.f;
-            int own = 0;                          // own batches accumulated in part[]
-            int first_b = 0;                      // first of them
-            for (int b = 0; b < nb; ++b) {
-                const int cnt = min(BATCH, n_up - b * BATCH);
-                if (NG > 1 && ((gbatch + b) % NG) != grp) { skip_n(BATCH); continue; }
-                uint4 q[BATCH][VPT];
-                fetch(q, cnt);
-                if (own == 0) first_b = b;
-#pragma unroll
-                for (int f = 0; f < FLUSH; ++f) {
-                    if (f == own) {               // uniform; keeps part[] statically indexed
-#pragma unroll
-                        for (int j = 0; j < BATCH; ++j) {
-                            float a0 = 0.f, a1 = 0.f;
-#pragma unroll
-                            for (int i = 0; i < VPT; ++i) E::dot(q[j][i], xq[i], a0, a1);
-                            part[f * BATCH + j] = a0 + a1;
-                        }
-                    }
-                }
-                ++own;
-                if (own == FLUSH || b + NG >= nb) {
-                    // two independent 8-value reductions (their shuffles interleave)
-                    float lo[8], hi[8];
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) { lo[j] = part[j]; hi[j] = part[8 + j]; }
-                    const float tot_lo = warp_reduce8(lo, lane);
-                    const float tot_hi = warp_reduce8(hi, lane);
-                    if ((lane & 3) == 0) {
-                        const int vi = ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);
-#pragma unroll
-                        for (int half = 0; half < 2; ++half) {
-                            const int pi = half * 8 + vi;                      // index in part[]
-                            const int f = pi / BATCH, j = pi % BATCH;          // own batch f of the window, item j
-                            const int item = (first_b + f * NG) * BATCH + j;   // position in the up phase
-                            if (f < own && item < n_up)
-                                red[((item % NMAT) * kGroupWarps + gw) * p.rmax + item / NMAT] = half ? tot_hi : tot_lo;
-                        }
-                    }
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) part[j] = 0.f;
-                    own = 0;
-                }
-            }
-            gbatch += nb;
-        }
-        named_bar_sync(1, NC);
-        for (int r = tid; r < nrows; r += NC) {
-            float u = 0.f;
-#pragma unroll
-            for (int w = 0; w < kGroupWarps; ++w) u += red[w * p.rmax + r];
-            float h;
-            if (GATED) {
-                float g = 0.f;
-#pragma unroll
-                for (int w = 0; w < kGroupWarps; ++w) g += red[(kGroupWarps + w) * p.rmax + r];
-                h = fmaxf(g, 0.f) * u;
-            } else {
-                if (ly.bup) u += E::load1(ly.bup, k0 + r);
-                h = fmaxf(u, 0.f);
-            }
-            h_s[r] = h;
-        }
-        named_bar_sync(1, NC);
-
-        // ------------------------------------------------------- down phase --
         float2 yacc[VPT][PAIRS];
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
-            const int v = gt + i * kGroupThreads;
+            const int v = tid + i * NC;
 #pragma unroll
             for (int c = 0; c < PAIRS; ++c) yacc[i][c] = make_float2(0.f, 0.f);
-            if (cta == 0 && grp == 0 && ly.bdown && v < nv) {   // the bias enters the sum exactly once
+            if (cta == 0 && ly.bdown && v < nv) {   // the bias enters the sum exactly once
 #pragma unroll
                 for (int c = 0; c < PAIRS; ++c)
                     yacc[i][c] = make_float2(E::load1(ly.bdown, v * EPV + 2 * c),
                                              E::load1(ly.bdown, v * EPV + 2 * c + 1));
             }
         }
-        {
-            const int nb = (nrows + BATCH - 1) / BATCH;
-            for (int b = 0; b < nb; ++b) {
-                const int cnt = min(BATCH, nrows - b * BATCH);
-                if (NG > 1 && ((gbatch + b) % NG) != grp) { skip_n(BATCH); continue; }
-                uint4 q[BATCH][VPT];
-                fetch(q, cnt);
+        float part[WIN];          // row sums of the current pair of batches (this thread's columns)
+#pragma unroll
+        for (int j = 0; j < WIN; ++j) part[j] = 0.f;
+
+        // One batch: its arithmetic, from the register buffer `q`.  `half` says which of the two
+        // buffers it is, i.e. which half of part[] an up batch fills.
+        auto process = [&](uint4 (&q)[BATCH][VPT], int b, const int H) {
+            if (b < nbu) {
+                // ------------------------------------------------ up (+ gate) rows --
 #pragma unroll
                 for (int j = 0; j < BATCH; ++j) {
-                    const float hk = (j < cnt) ? h_s[b * BATCH + j] : 0.f;
+                    float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+                    for (int i = 0; i < VPT; ++i) E::dot(q[j][i], xq[i], a0, a1);
+                    part[H * BATCH + j] = a0 + a1;
+                }
+                if (H == 1 || b == nbu - 1) {
+                    // the pair of batches is complete (or the phase ends on its first half, whose
+                    // second half then holds stale sums of rows that do not exist: not stored)
+                    const float tot = warp_reduce_n(part, lane);
+                    const int vi = WIN == 8 ? ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1)
+                                            : ((lane >> 4) & 1) * 2 + ((lane >> 3) & 1);
+                    const int item = (b - H) * BATCH + vi;           // position in the up phase
+                    if ((lane & (32 / WIN - 1)) == 0 && item < n_up)
+                        red[((item % NMAT) * nwarps + warp) * p.rmax + item / NMAT] = tot;
+                }
+                if (b == nbu - 1) {
+                    CI_STAMP(stamps, sb, 1);
+                    named_bar_sync(1, NC);
+                    for (int r = tid; r < nrows; r += NC) {
+                        float u = 0.f;
+                        for (int w = 0; w < nwarps; ++w) u += red[w * p.rmax + r];
+                        float h;
+                        if (GATED) {
+                            float g = 0.f;
+                            for (int w = 0; w < nwarps; ++w) g += red[(nwarps + w) * p.rmax + r];
+                            h = fmaxf(g, 0.f) * u;
+                        } else {
+                            if (ly.bup) u += E::load1(ly.bup, k0 + r);
+                            h = fmaxf(u, 0.f);
+                        }
+                        h_s[r] = h;
+                    }
+                    named_bar_sync(1, NC);
+                    CI_STAMP(stamps, sb, 2);
+                }
+            } else {
+                // ------------------------------------------------------- down rows --
+                const int r0 = (b - nbu) * BATCH;
+#pragma unroll
+                for (int j = 0; j < BATCH; ++j) {
+                    const float hk = (r0 + j < nrows) ? h_s[r0 + j] : 0.f;
                     if (hk != 0.f) {                              // uniform: ReLU zeros cost no arithmetic
                         const float2 hh = make_float2(hk, hk);
 #pragma unroll
@@ -543,88 +529,84 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
                     }
                 }
             }
-            gbatch += nb;
+        };
+
+        {
+            uint4 qa[BATCH][VPT], qb[BATCH][VPT];
+            if (nbt > 0) fetch(qa);
+            for (int b = 0; b < nbt; b += 2) {
+                if (b + 1 < nbt) fetch(qb);
+                process(qa, b, 0);
+                if (b + 2 < nbt) fetch(qa);
+                if (b + 1 < nbt) process(qb, b + 1, 1);
+            }
+            if (nbt == 0) {                          // a CTA without neurons still meets the others at the barriers
+                named_bar_sync(1, NC);
+                named_bar_sync(1, NC);
+            }
         }
+        CI_STAMP(stamps, sb, 3);
 
         // ----------------------------------------- cross-CTA sum of partial y --
         // Every CTA adds its partial into the layer's target; after the grid barrier every CTA
         // reads the sum back.  Targets rotate over three buffers: while layer l's is read, the
         // one layer l+2 will use is cleared (last read before the barrier of l).
         const bool last = (l == p.L - 1);
-        float* ybase = p.ybuf + (size_t)(l % kYBuffers) * kYCopies * d;
-        float* ytarget = ybase + (size_t)(cta & (kYCopies - 1)) * d;
-        // One sum per CTA leaves the chip, as one bulk reduction: group 1 hands its partial to
-        // group 0 through shared memory, group 0 leaves the CTA's partial there, and the copy
-        // engine adds the whole vector into the target (L2 then sees 128-byte line reductions
-        // instead of a thousand 16-byte atomics per CTA, whose acknowledgements a fence had to
-        // wait for).
-        if (NG == 2) {
-            if (grp == 1) {
+        float* ytarget = p.ybuf + (size_t)(l % kYBuffers) * d;
+        // One sum per CTA leaves the chip, as one bulk reduction from shared memory (L2 then
+        // sees 128-byte line reductions instead of a thousand 16-byte atomics per CTA).
 #pragma unroll
-                for (int i = 0; i < VPT; ++i)
+        for (int i = 0; i < VPT; ++i) {
+            const int v = tid + i * NC;
+            if (v < nv) {
 #pragma unroll
-                    for (int c = 0; c < PAIRS; c += 2)
-                        *reinterpret_cast<float4*>(ysum + (size_t)(gt + i * kGroupThreads) * EPV + 2 * c) =
-                            make_float4(yacc[i][c].x, yacc[i][c].y, yacc[i][c + 1].x, yacc[i][c + 1].y);
+                for (int c = 0; c < PAIRS; c += 2)
+                    *reinterpret_cast<float4*>(ysum + (size_t)v * EPV + 2 * c) =
+                        make_float4(yacc[i][c].x, yacc[i][c].y, yacc[i][c + 1].x, yacc[i][c + 1].y);
             }
-            named_bar_sync(1, NC);
         }
-        if (grp == 0) {
-#pragma unroll
-            for (int i = 0; i < VPT; ++i) {
-#pragma unroll
-                for (int c = 0; c < PAIRS; c += 2) {
-                    float4* cell = reinterpret_cast<float4*>(ysum + (size_t)(gt + i * kGroupThreads) * EPV + 2 * c);
-                    float4 t = make_float4(yacc[i][c].x, yacc[i][c].y, yacc[i][c + 1].x, yacc[i][c + 1].y);
-                    if (NG == 2) {
-                        const float4 o = *cell;
-                        t.x += o.x; t.y += o.y; t.z += o.z; t.w += o.w;
-                    }
-                    *cell = t;
-                }
-            }
-            fence_proxy_async();          // these generic-proxy writes are read by the copy engine next
-        }
+        fence_proxy_async();          // these generic-proxy writes are read by the copy engine next
         named_bar_sync(1, NC);
         // One thread runs the exchange: the CTA's reduction and the wait for its completion, the
         // arrival at the grid barrier (a release: the CTA's earlier plain writes to global memory,
         // such as the cleared target of a later layer, are known to this thread through the CTA
         // barriers since), the wait for everybody else's arrival, and the copy that brings the
-        // sum back; the other consumers sleep on that copy's barrier.  The sum comes back as one
-        // bulk copy into the buffer the partial left from (256 requests of 128 bytes per CTA
-        // instead of some thousand 16-byte loads).
+        // sum back into the buffer the partial left from; the other consumers sleep on that
+        // copy's barrier.
         if (tid == 0) {
+            CI_STAMP(stamps, sb, 4);
             if (!*abort_flag) {
                 bulk_reduce_add_f32(ytarget, smem_u32(ysum), (uint32_t)d * (uint32_t)sizeof(float));
                 bulk_wait_all();
-                grid_arrive_and_wait(p.ctrl, (unsigned)(l + 1) * (unsigned)G, abort_flag);
+                CI_STAMP(stamps, sb, 5);
+                red_release_add(&p.ctrl[1], 1u);
+                *arrived = l + 1;         // the fence is behind us: the producer may trickle
+                CI_STAMP(stamps, sb, 6);
+                grid_wait(p.ctrl, (unsigned)(l + 1) * (unsigned)G, abort_flag);
+                CI_STAMP(stamps, sb, 7);
             }
             if (!*abort_flag) {
                 const uint32_t yb = smem_u32(y_bar);
-                mbar_arrive_expect_tx(yb, (uint32_t)(kYCopies * d) * (uint32_t)sizeof(float));
-                bulk_g2s(smem_u32(ysum), ybase, (uint32_t)(kYCopies * d) * (uint32_t)sizeof(float), yb);
+                mbar_arrive_expect_tx(yb, (uint32_t)d * (uint32_t)sizeof(float));
+                bulk_g2s(smem_u32(ysum), ytarget, (uint32_t)d * (uint32_t)sizeof(float), yb);
                 *layers_done = l + 1;     // the exchange's last request is on its way: the producer may go on
             }
         }
         wait_slot(smem_u32(y_bar), (uint32_t)(l & 1), abort_flag, p.ctrl);
+        CI_STAMP(stamps, sb, 8);
 
         // ------------------------- next input: (x + y) / rms(x + y), rounded --
         float ssp[4] = {0.f, 0.f, 0.f, 0.f};   // four chains of the sum of squares
         float2 xn[VPT][PAIRS];        // x + y in fp32, until the norm is known
-        const bool writer = (cta == l % G) && grp == 0;   // the CTA that stores this layer's y
+        const bool writer = (cta == l % G);   // the CTA that stores this layer's y
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
-            const int v = gt + i * kGroupThreads;
+            const int v = tid + i * NC;
             E::unpack(xq[i], xn[i]);
             if (v < nv) {
 #pragma unroll
                 for (int c = 0; c < PAIRS; c += 2) {
-                    float4 t = *reinterpret_cast<const float4*>(ysum + (size_t)v * EPV + 2 * c);
-#pragma unroll
-                    for (int cp = 1; cp < kYCopies; ++cp) {
-                        const float4 o = *reinterpret_cast<const float4*>(ysum + (size_t)cp * d + (size_t)v * EPV + 2 * c);
-                        t.x += o.x; t.y += o.y; t.z += o.z; t.w += o.w;
-                    }
+                    const float4 t = *reinterpret_cast<const float4*>(ysum + (size_t)v * EPV + 2 * c);
                     if (writer) {
                         if (p.y_layers) *reinterpret_cast<float4*>(p.y_layers + (size_t)l * d + (size_t)v * EPV + 2 * c) = t;
                         if (last) *reinterpret_cast<float4*>(p.y_last + (size_t)v * EPV + 2 * c) = t;
@@ -643,57 +625,49 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
         }
         float ss = (ssp[0] + ssp[1]) + (ssp[2] + ssp[3]);
         {   // clear the target that layer l + 2 will use
-            float4* z = reinterpret_cast<float4*>(p.ybuf + (size_t)((l + 2) % kYBuffers) * kYCopies * d);
-            const int n4 = kYCopies * d / 4;
+            float4* z = reinterpret_cast<float4*>(p.ybuf + (size_t)((l + 2) % kYBuffers) * d);
+            const int n4 = d / 4;
             for (int i = cta * NC + tid; i < n4; i += G * NC) z[i] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        if (last) break;
-        // every group holds all columns, so each forms the norm on its own (same sums, same order)
+        if (last) { CI_STAMP(stamps, sb, 9); break; }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-        if (lane == 0) ss_red[grp * kGroupWarps + gw] = ss;
-        named_bar_sync(2 + grp, kGroupThreads);
+        if (lane == 0) ss_red[warp] = ss;
+        named_bar_sync(1, NC);
         float tot = 0.f;
-#pragma unroll
-        for (int w = 0; w < kGroupWarps; ++w) tot += ss_red[grp * kGroupWarps + w];
+        for (int w = 0; w < nwarps; ++w) tot += ss_red[w];
         const float inv = rsqrtf(tot * p.inv_d);     // within 2 ulp of 1 / sqrt(mean square)
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
-            const int v = gt + i * kGroupThreads;
+            const int v = tid + i * NC;
 #pragma unroll
             for (int c = 0; c < PAIRS; ++c) {
                 xn[i][c].x *= inv;
                 xn[i][c].y *= inv;
             }
-            xq[i] = E::pack(xn[i]);       // rounds to the layer-input type
-            if (p.x_layers && cta == (l + 1) % G && grp == 0 && v < nv)
+            xq[i] = v < nv ? E::pack(xn[i]) : make_uint4(0, 0, 0, 0);       // rounds to the layer-input type
+            if (p.x_layers && cta == (l + 1) % G && v < nv)
                 reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(p.x_layers) +
                                          (size_t)(l + 1) * p.row_bytes)[v] = xq[i];
         }
+        CI_STAMP(stamps, sb, 9);
     }
 }
 
 // ------------------------------------------------------------------- host ---
-// fp32 buffer in which the CTA's partial y is assembled: every thread of a group stores all its columns
-static size_t ysum_smem_bytes(int groups, int vpt, size_t esize)
+static size_t fixed_smem_bytes(int rmax, bool gated, int nwarps)
 {
-    (void)groups;
-    return (size_t)kYCopies * vpt * kGroupThreads * (16 / esize) * sizeof(float);   // room for the copies read back
-}
-
-static size_t fixed_smem_bytes(int rmax, bool gated, int groups)
-{
-    size_t b = (2 * kMaxSlots + 2) * sizeof(uint64_t);
-    b += (size_t)(gated ? 2 : 1) * kGroupWarps * rmax * sizeof(float);
-    b += (size_t)rmax * sizeof(float);
-    b += (size_t)groups * kGroupWarps * sizeof(float) + 16;
+    size_t b = (2 * kMaxBatchSlots + 2) * sizeof(uint64_t);
+    b += (size_t)(gated ? 2 : 1) * nwarps * rmax * sizeof(float);      // red
+    b += (size_t)rmax * sizeof(float);                                 // h_s
+    b += (size_t)kMaxWarps * sizeof(float) + 16;                       // ss_red, flags
     return (b + 127) & ~(size_t)127;
 }
 
-template <typename T, int NG, int VPT, bool GATED>
+template <typename T, int VPT, bool GATED>
 static coreinfer_status launch_one(const DecodeParams& p, int grid, size_t smem, cudaStream_t st)
 {
-    auto kern = decode_stack_kernel<T, NG, VPT, GATED>;
+    auto kern = decode_stack_kernel<T, VPT, GATED>;
     static thread_local size_t configured[64] = {0};
     int dev = 0;
     CI_CUDA(cudaGetDevice(&dev));
@@ -703,7 +677,7 @@ static coreinfer_status launch_one(const DecodeParams& p, int grid, size_t smem,
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3((unsigned)(NG * kGroupThreads + 32));
+    cfg.blockDim = dim3((unsigned)(p.nc + 32));
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -716,7 +690,7 @@ static coreinfer_status launch_one(const DecodeParams& p, int grid, size_t smem,
 }
 
 // Debugging aid: COREINFER_RING_SLOTS=n in the environment (read once) caps the ring of the
-// batch-1 stack kernel at n slots, so that tests can make the ring wrap every few rows.
+// batch-1 stack kernel at n rows, so that tests can make the ring wrap every few rows.
 static int ring_slots_cap()
 {
     static const int cap = [] {
@@ -726,24 +700,12 @@ static int ring_slots_cap()
     return cap;
 }
 
-static int groups_for(int nv) { return nv <= 2 * kGroupThreads ? 2 : 1; }
-static int vpt_for(int nv)
-{
-    const int v = (nv + kGroupThreads - 1) / kGroupThreads;
-    return v <= 1 ? 1 : v <= 2 ? 2 : v <= 3 ? 3 : v <= 5 ? 5 : 8;
-}
-
 template <typename T, bool GATED>
-static coreinfer_status launch_shape(int groups, int vpt, const DecodeParams& p, int grid, size_t smem,
-                                     cudaStream_t st)
+static coreinfer_status launch_shape(int vpt, const DecodeParams& p, int grid, size_t smem, cudaStream_t st)
 {
-    if (groups == 2) {
-        if (vpt <= 1) return launch_one<T, 2, 1, GATED>(p, grid, smem, st);
-        return launch_one<T, 2, 2, GATED>(p, grid, smem, st);
-    }
-    if (vpt <= 3) return launch_one<T, 1, 3, GATED>(p, grid, smem, st);
-    if (vpt <= 5) return launch_one<T, 1, 5, GATED>(p, grid, smem, st);
-    return launch_one<T, 1, 8, GATED>(p, grid, smem, st);
+    if (vpt <= 1) return launch_one<T, 1, GATED>(p, grid, smem, st);
+    if (vpt == 2) return launch_one<T, 2, GATED>(p, grid, smem, st);
+    return launch_one<T, 3, GATED>(p, grid, smem, st);
 }
 
 static coreinfer_status check_common(const void* x, int batch, coreinfer_dtype dtype,
@@ -774,9 +736,10 @@ static coreinfer_status check_layer(const coreinfer_layer& ly, int l, coreinfer_
     return COREINFER_OK;
 }
 
+
 static size_t b1_workspace_bytes(int d_model)
 {
-    return kCtrlBytes + (size_t)kYBuffers * kYCopies * (size_t)d_model * sizeof(float);
+    return kCtrlBytes + (size_t)kYBuffers * (size_t)d_model * sizeof(float);
 }
 
 // Shared by the one-layer and the stack entry points (batch 1).
@@ -819,47 +782,53 @@ static coreinfer_status decode_stack_b1(const coreinfer_layer* layers, int L, co
     if ((unsigned long long)Kmax * (unsigned long long)G >= (1ull << 32))
         CI_FAIL(COREINFER_ERR_UNSUPPORTED, "K = %d is too large for the slab split (K * SM count must stay below 2^32)", Kmax);
     p.inv_d = 1.0f / (float)d_model;
-    const int groups = groups_for(p.nv);
-    if ((p.nv + kGroupThreads - 1) / kGroupThreads > 8)
+    // Consumer threads: every thread owns `vpt` 16-byte vectors of a row; as many warps as the
+    // row needs, 16 at most.
+    const int vpt = (p.nv + kMaxConsumers - 1) / kMaxConsumers;
+    if (vpt > kMaxVpt)
         CI_FAIL(COREINFER_ERR_UNSUPPORTED, "d_model %d is too wide for this kernel (max %d bytes per row)",
-                d_model, 8 * kGroupThreads * 16);
-    const int vpt = groups == 2 ? ((p.nv + kGroupThreads - 1) / kGroupThreads <= 1 ? 1 : 2) : vpt_for(p.nv);
-    const int batch = batch_for(groups, groups == 2 ? vpt : (vpt <= 3 ? 3 : vpt));
-    const size_t fixed0 = fixed_smem_bytes(p.rmax, gated, groups);
-    const size_t fixed = fixed0 + ysum_smem_bytes(groups, vpt, esize);
-    if (fixed + (size_t)batch * p.slot_bytes > (size_t)di.smem_optin)
+                d_model, kMaxVpt * max_consumers(kMaxVpt) * 16);
+    p.nc = (((p.nv + vpt - 1) / vpt) + 31) & ~31;
+    if (p.nc > max_consumers(vpt))
+        CI_FAIL(COREINFER_ERR_UNSUPPORTED, "d_model %d is too wide for this kernel (max %d bytes per row)",
+                d_model, kMaxVpt * max_consumers(kMaxVpt) * 16);
+    const int batch = batch_for(vpt);
+    const size_t bslot_bytes = (size_t)batch * p.slot_bytes;
+    const size_t fixed0 = fixed_smem_bytes(p.rmax, gated, p.nc / 32);
+    const size_t fixed = fixed0 + (((size_t)d_model * sizeof(float) + 127) & ~(size_t)127);    // + the partial y / the sum
+    long long bslots = ((long long)di.smem_optin - (long long)fixed) / (long long)bslot_bytes;
+    if (bslots > kMaxBatchSlots) bslots = kMaxBatchSlots;
+    if (ring_slots_cap() > 0 && bslots > ring_slots_cap() / batch) bslots = ring_slots_cap() / batch;
+    if (bslots < 2)
         CI_FAIL(COREINFER_ERR_UNSUPPORTED, "K = %d, d_model = %d do not fit in shared memory", Kmax, d_model);
-    long long slots = ((long long)di.smem_optin - (long long)fixed) / p.slot_bytes;
-    if (slots > kMaxSlots) slots = kMaxSlots;
-    if (ring_slots_cap() > 0 && slots > ring_slots_cap()) slots = ring_slots_cap();
-    // With two groups a slot must always come back to the same group (a group never waits on the
-    // other's items, so only then can it never be a full ring pass ahead of a barrier it tests):
-    // every batch takes `batch` slots and the ring holds a whole number of batch pairs.
-    if (groups == 2) slots -= slots % (2 * batch);
-    if (slots < (long long)groups * batch)
-        CI_FAIL(COREINFER_ERR_UNSUPPORTED, "the ring of %lld slots is smaller than %d batches of %d rows", slots,
-                groups, batch);
-    p.n_slots = (int)slots;
-    const size_t smem = fixed + (size_t)p.n_slots * p.slot_bytes;
-    // Measured on the four model shapes: about 100 KB of the next layer requested ahead of the
-    // exchange is best (12 rows of 8 or 10 KB; 4-5 rows of 18 KB); more delays the exchange's own
-    // messages, less leaves the ring empty when the consumers come back.
-    p.runahead = p.slot_bytes <= 12 * 1024 ? 12 : (96 * 1024 / p.slot_bytes < 4 ? 4 : 96 * 1024 / p.slot_bytes);
-    p.ysum_ofs = (int)((size_t)p.n_slots * p.slot_bytes + fixed0);
+    p.n_bslots = (int)bslots;
+    const size_t smem = fixed + (size_t)p.n_bslots * bslot_bytes;
+    // While an exchange is on, the next layer's rows are requested in two parts (measured on the
+    // four model shapes): about 72 KB ahead of the exchange -- more would still be in flight when
+    // the CTA's fence runs, and a fence waits for the SM's own copies in flight -- and the rest of
+    // the ring after the CTA's arrival, one batch per 1400 cycles and 32 KB, which is about the pace
+    // at which HBM serves one SM.
+    const int rows_ahead = 72 * 1024 / p.slot_bytes;
+    p.runahead = rows_ahead / batch < 1 ? 1 : rows_ahead / batch;
+    if (p.runahead > p.n_bslots) p.runahead = p.n_bslots;
+    p.trickle = p.n_bslots - p.runahead;
+    p.trickle_gap = (int)(1400ll * (long long)bslot_bytes / 32768);
+    p.ysum_ofs = (int)((size_t)p.n_bslots * bslot_bytes + fixed0);
     p.x0 = x0;
     p.y_last = y_last;
     p.y_layers = y_layers;
     p.x_layers = x_layers;
     p.ctrl = (unsigned*)workspace;
     p.ybuf = (float*)((uint8_t*)workspace + kCtrlBytes);
+    p.stamps = stamps_buffer((size_t)G * L * kStampSlots * sizeof(unsigned long long));
 
     // Control words and the reduction targets start at zero.
     CI_CUDA(cudaMemsetAsync(workspace, 0, b1_workspace_bytes(d_model), st));
     if (dtype == COREINFER_BF16)
-        return gated ? launch_shape<__nv_bfloat16, true>(groups, vpt, p, G, smem, st)
-                     : launch_shape<__nv_bfloat16, false>(groups, vpt, p, G, smem, st);
-    return gated ? launch_shape<float, true>(groups, vpt, p, G, smem, st)
-                 : launch_shape<float, false>(groups, vpt, p, G, smem, st);
+        return gated ? launch_shape<__nv_bfloat16, true>(vpt, p, G, smem, st)
+                     : launch_shape<__nv_bfloat16, false>(vpt, p, G, smem, st);
+    return gated ? launch_shape<float, true>(vpt, p, G, smem, st)
+                 : launch_shape<float, false>(vpt, p, G, smem, st);
 }
 
 // decode_batch.cu
