@@ -42,6 +42,9 @@ def parse_args():
     ap.add_argument("--no-dense", action="store_true", help="skip the dense (alpha = beta = 1) comparison")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-configs", action="store_true",
+                    help="skip the per-configuration block (decode, dense, selection and compaction timings of the "
+                         "other workload shapes, measured after the timed region)")
     ap.add_argument("--no-graph", action="store_true", help="issue every call from the host instead of replaying CUDA graphs")
     ap.add_argument("--decode-only", type=int, default=0, metavar="LAYERS",
                     help="profiling target: only decode launches through the first LAYERS layers of the config "
@@ -487,11 +490,115 @@ def run_ours(args, cfg):
         "clocks": clocks, "wall_s": wall,
         "context": "paper (TITAN Xp, end to end, other workload): 10.33x over HuggingFace, 2.72x over PowerInfer",
     }
+    if not args.no_configs and world == 1:
+        del weights, acts, stack
+        torch.cuda.empty_cache()
+        line["configs"] = other_configs(ci, wl, peak, cfg.name)
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = oracle_sample(cfg, n_layers=4, n_tokens=min(cfg.decode_steps, 256))
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+# ------------------------------------------------- the other configurations ---
+def _time_ms(fn, stream, reps):
+    import torch
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    fn(); torch.cuda.synchronize()
+    a.record(stream)
+    for _ in range(reps): fn()
+    b.record(stream); torch.cuda.synchronize()
+    return a.elapsed_time(b) / reps
+
+
+def decode_stack_rate(ci, wl, cfg, K, layers, batch, peak, tokens=16, reps=3):
+    """Decode launches alone through `layers` layers of random compacted [K, d] weights of cfg's shape
+    (the decode stage does not care how the rows were chosen); rates are per full stack of cfg.L layers,
+    scaled from the cut by the layer count when layers < cfg.L."""
+    import torch
+    cut = cfg.with_(L=layers)
+    w = [wl.compacted_weights_random(cut, l, K, device="cuda") for l in range(layers)]
+    arr = ci.binding.make_layers([(u, g, dn, None, None) for (u, g, dn) in w])
+    kind = ci.FFN_RELU_GATED if cfg.gated else ci.FFN_RELU
+    xs = [wl.decode_input(cfg, s, device="cuda", batch=batch) for s in range(tokens)]
+    y = torch.empty((batch, cfg.d_model), device="cuda")
+    ws = torch.empty(ci.coreinfer_ffn_decode_stack_workspace_bytes(layers, batch, cfg.d_model, K), dtype=torch.uint8,
+                     device="cuda")
+    stream = torch.cuda.current_stream()
+    ms = _time_ms(lambda: [ci.coreinfer_ffn_decode_stack(arr, xs[t], kind, y, None, None, ws, stream) for t in range(tokens)],
+                  stream, reps) / tokens
+    ci.coreinfer_workspace_status(ws)
+    nbytes = layers * cfg.n_mat * K * cfg.d_model * cfg.esize
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    full_ms = ms * cfg.L / layers
+    out = {"K": K, "batch": batch, "layers_timed": layers, "us_per_layer": 1e3 * ms / layers, "gbs": gbs,
+           "frac_of_measured": gbs / peak, "frac_of_8TBs": gbs / 8000.0,
+           "steps_per_s_full_stack": 1e3 / full_ms, "sequence_tok_s_full_stack": batch * 1e3 / full_ms,
+           "launches_timed": tokens * reps}
+    del w, arr
+    return out
+
+
+def prefill_stage_times(ci, wl, cfg, T, beta, layer=0):
+    """Selection and compaction of ONE full-size layer of cfg: microseconds per layer."""
+    import torch
+    kind = ci.FFN_RELU_GATED if cfg.gated else ci.FFN_RELU
+    w_up, w_gate, w_down = wl.layer_weights(cfg, layer, device="cuda")
+    if cfg.planted:
+        A, _ = wl.planted_activations(cfg, layer, T, device="cuda")
+    else:
+        X = wl.prompt_hidden(cfg, device="cuda", T=T)
+        A = torch.empty((T, cfg.d_ff), device="cuda")
+        ci.coreinfer_ffn_dense_ref(X, kind, w_up, w_gate, w_down, None, None, A, None)
+    K = ci.coreinfer_count(beta, cfg.d_ff)
+    S = torch.empty(K, dtype=torch.int32, device="cuda")
+    ws = torch.empty(ci.coreinfer_select_workspace_bytes(T, cfg.d_ff), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+    sel = _time_ms(lambda: ci.coreinfer_select_core(A, cfg.alpha, beta, S, None, ws, stream), stream, 10)
+    new = lambda: torch.empty((K, cfg.d_model), dtype=cfg.torch_dtype, device="cuda")
+    up_c, down_c, gate_c = new(), new(), (new() if cfg.gated else None)
+    cmp_ = _time_ms(lambda: ci.coreinfer_compact(w_up, w_gate, w_down, None, S, K, up_c, gate_c, down_c, None, stream),
+                    stream, 5)
+    return {"T": T, "K": K, "select_us": 1e3 * sel, "select_floor_us_at_measured_peak": None,
+            "activation_bytes": 4 * T * cfg.d_ff, "compact_us": 1e3 * cmp_}
+
+
+def other_configs(ci, wl, peak, headline):
+    """Decode rates (sparse and dense), selection and compaction times of every workload
+    configuration other than the headline one; CUDA events, outside the timed region."""
+    import torch
+    out = {}
+    for name in ("opt125m-1layer", "opt13b", "relu-llama2-7b", "opt66b"):
+        if name == headline:
+            continue
+        cfg = wl.CONFIGS[name]
+        block = {"dtype": cfg.dtype, "L": cfg.L, "d_model": cfg.d_model, "d_ff": cfg.d_ff, "gated": cfg.gated}
+        # the OPT-66B-shaped stack is timed on a cut (its 64 compacted layers hold 17 GB, its dense ones 87 GB)
+        layers = 16 if name == "opt66b" else cfg.L
+        betas = wl.OPT13B_BETAS if name == "opt13b" else (cfg.beta,)
+        block["decode"] = {}
+        for beta in betas:
+            K = ci.coreinfer_count(beta, cfg.d_ff)
+            tokens = 16 if K * cfg.d_model * layers < 4e9 else 4
+            block["decode"]["beta=%g" % beta] = decode_stack_rate(ci, wl, cfg, K, layers, 1, peak, tokens=tokens)
+            torch.cuda.empty_cache()
+        if 1.0 not in betas:
+            dl = min(layers, 16)
+            block["dense"] = decode_stack_rate(ci, wl, cfg, cfg.d_ff, dl, 1, peak, tokens=4, reps=2)
+            torch.cuda.empty_cache()
+        if name == "relu-llama2-7b":
+            K = ci.coreinfer_count(cfg.beta, cfg.d_ff)
+            block["decode"]["beta=%g, 8 sequences" % cfg.beta] = decode_stack_rate(ci, wl, cfg, K, layers, 8, peak)
+        Ts = wl.OPT66B_TS if name == "opt66b" else (cfg.T,)
+        block["prefill"] = []
+        for T in Ts:
+            r = prefill_stage_times(ci, wl, cfg, T, cfg.beta)
+            r["select_floor_us_at_measured_peak"] = r["activation_bytes"] / peak / 1e3
+            block["prefill"].append(r)
+            torch.cuda.empty_cache()
+        out[name] = block
+    return out
 
 
 def run_decode_only(args, cfg):
