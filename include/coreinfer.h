@@ -118,6 +118,19 @@ coreinfer_status coreinfer_compact(const void* w_up, const void* w_gate, const v
                                    void* w_up_c, void* w_gate_c, void* w_downT_c, void* b_up_c,
                                    void* cuda_stream);
 
+/* Checks a core index list before it is used: coreinfer_compact trusts `core_idx` (its gather
+ * kernels read the weights at those indices without a bounds test), so a list that does not
+ * come from coreinfer_select_core should pass through here first.  (A helper of the boundary;
+ * the paper has no counterpart.)  Enqueues one small kernel that writes
+ *   report[0] = number of positions k with core_idx[k] outside [0, d_ff) or not greater than
+ *               core_idx[k-1] (the list must be strictly ascending),
+ *   report[1] = the first such position, INT32_MAX if there is none,
+ * to `report` (device, two int32); the caller reads them back once the stream has reached that
+ * point.  Only core_idx[0 .. K) is read.
+ * Errors: INVALID_ARG, CUDA. */
+coreinfer_status coreinfer_verify_core_idx(const int32_t* core_idx, int32_t K, int32_t d_ff,
+                                           int32_t* report, void* cuda_stream);
+
 /* ------------------------------------------------------------------ (3) --
  * Decode FFN over compacted weights (Section 4.2), one layer:
  *   h_k = act(w_up_c[k,:] . x (+ b_up_c[k]))   [gated: max(w_gate_c[k,:] . x, 0) * (w_up_c[k,:] . x)]
@@ -201,7 +214,8 @@ coreinfer_status coreinfer_ffn_decode_stack(const coreinfer_layer* layers, int32
  * gives up 128 KiB for the life of the process, and the call itself allocates nothing (no
  * cudaMalloc / cudaFree, no allocating library routine).
  *
- * Arguments and results are those of coreinfer_ffn_decode_stack without the workspace pair.
+ * Arguments and results are those of coreinfer_ffn_decode_stack without the workspace pair,
+ * for batch 1 only (any other batch returns COREINFER_ERR_UNSUPPORTED).
  * Limit: the scratch the kernel needs, 256 + 12 * d_model bytes (any number of layers), must fit
  * in 128 KiB, i.e. d_model <= 10901; wider models return COREINFER_ERR_UNSUPPORTED and enqueue
  * nothing -- use the workspace variant for them.

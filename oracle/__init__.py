@@ -23,22 +23,25 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "coreinfer_oracle.c")
 _LIB = os.path.join(_HERE, "_build", "libcoreinfer_oracle.so")
+_LIB_F32 = os.path.join(_HERE, "_build", "libcoreinfer_oracle_f32acc.so")   # -DORACLE_F32_ACC, not the oracle
 _lock = threading.Lock()
 _lib = None
 
 
-def build(force: bool = False) -> str:
-    """Compile the oracle with gcc (no fast-math) and return the library path."""
-    os.makedirs(os.path.dirname(_LIB), exist_ok=True)
-    if (not force and os.path.exists(_LIB)
-            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
-        return _LIB
-    tmp = _LIB + ".tmp.%d" % os.getpid()
+def build(force: bool = False, f32_acc: bool = False) -> str:
+    """Compile the oracle with gcc (C11, -O2, OpenMP, no fast-math, no contraction) and
+    return the library path.  f32_acc builds the fp32-accumulator variant of the FFN loops."""
+    lib = _LIB_F32 if f32_acc else _LIB
+    os.makedirs(os.path.dirname(lib), exist_ok=True)
+    if (not force and os.path.exists(lib)
+            and os.path.getmtime(lib) >= os.path.getmtime(_SRC)):
+        return lib
+    tmp = lib + ".tmp.%d" % os.getpid()
     cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp",
-           "-fno-fast-math", "-ffp-contract=off", "-o", tmp, _SRC, "-lm"]
+           "-fno-fast-math", "-ffp-contract=off"] + (["-DORACLE_F32_ACC"] if f32_acc else []) + ["-o", tmp, _SRC, "-lm"]
     subprocess.run(cmd, check=True)
-    os.replace(tmp, _LIB)
-    return _LIB
+    os.replace(tmp, lib)
+    return lib
 
 
 def _load():
@@ -132,6 +135,32 @@ def compact(w_up, w_gate, w_down, b_up, S):
                            dt.itemsize, d, N, _ptr(S), K,
                            _ptr(up_c), _ptr(gate_c), _ptr(down_c), _ptr(bup_c))
     return up_c, gate_c, down_c, bup_c
+
+
+_lib_f32 = None
+
+
+def ffn_f32_accumulators(x, kind, w_up_c, w_gate_c, w_downT_c, b_up_c=None, b_down=None):
+    """The FFN loops of ffn() with fp32 running sums (the -DORACLE_F32_ACC build).  Not the
+    oracle: it exists to report the distance between fp32 and double accumulation."""
+    global _lib_f32
+    with _lock:
+        if _lib_f32 is None:
+            _lib_f32 = ctypes.CDLL(build(f32_acc=True))
+            vp, i32 = ctypes.c_void_p, ctypes.c_int32
+            _lib_f32.oracle_ffn.restype = None
+            _lib_f32.oracle_ffn.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+    x = _f32(x)
+    if x.ndim == 1:
+        x = x[None, :]
+    B, d = x.shape
+    w_up_c, w_gate_c, w_downT_c = _f32(w_up_c), _f32(w_gate_c), _f32(w_downT_c)
+    b_up_c, b_down = _f32(b_up_c), _f32(b_down)
+    K = w_up_c.shape[0]
+    y = np.empty((B, d), dtype=np.float32)
+    _lib_f32.oracle_ffn(_ptr(x), B, int(kind), d, K, _ptr(w_up_c), _ptr(w_gate_c), _ptr(w_downT_c),
+                        _ptr(b_up_c), _ptr(b_down), _ptr(y), None)
+    return y
 
 
 def ffn(x, kind, w_up_c, w_gate_c, w_downT_c, b_up_c=None, b_down=None, return_h=False):

@@ -29,6 +29,9 @@
  *
  * Floating point: tensors are stored as fp32 (bf16 inputs are widened exactly
  * by the caller); every running sum is a double and is rounded to fp32 once.
+ * Compiled with -DORACLE_F32_ACC the running sums of oracle_ffn are fp32 instead
+ * (plain sequential fp32 sums): that variant is not the oracle, it only serves
+ * to report how far a pure fp32 accumulation is from the double one.
  *
  * Every function here is pinned by tests that do not call it to produce their
  * expected values (hand-worked example, brute-force ranking, library sort and
@@ -38,6 +41,12 @@
 #include <stdlib.h>
 #include <string.h>
 #include <math.h>
+
+#ifdef ORACLE_F32_ACC
+typedef float acc_t;
+#else
+typedef double acc_t;
+#endif
 #ifdef _OPENMP
 #include <omp.h>
 #endif
@@ -187,38 +196,46 @@ void oracle_ffn(const float *x, int32_t B, int32_t kind, int32_t d, int32_t K,
                 const float *b_up_c, const float *b_down, float *y, float *h_out)
 {
     float *h = (float *)malloc(sizeof(float) * (size_t)(K > 0 ? K : 1));
-    double *acc = (double *)malloc(sizeof(double) * (size_t)(d > 0 ? d : 1));
+    acc_t *acc = (acc_t *)malloc(sizeof(acc_t) * (size_t)(d > 0 ? d : 1));
     for (int32_t b = 0; b < B; ++b) {
         const float *xb = x + (size_t)b * d;
 #ifdef _OPENMP
 #pragma omp parallel for schedule(static)
 #endif
         for (int32_t k = 0; k < K; ++k) {
-            double su = 0.0;
+            acc_t su = 0;
             for (int32_t i = 0; i < d; ++i)
-                su += (double)w_up_c[(size_t)k * d + i] * (double)xb[i];
-            if (kind == 0 && b_up_c) su += (double)b_up_c[k];
+                su += (acc_t)w_up_c[(size_t)k * d + i] * (acc_t)xb[i];
+            if (kind == 0 && b_up_c) su += (acc_t)b_up_c[k];
             float u = (float)su;
             if (kind == 1) {
-                double sg = 0.0;
+                acc_t sg = 0;
                 for (int32_t i = 0; i < d; ++i)
-                    sg += (double)w_gate_c[(size_t)k * d + i] * (double)xb[i];
+                    sg += (acc_t)w_gate_c[(size_t)k * d + i] * (acc_t)xb[i];
                 float g = (float)sg;
                 h[k] = (g > 0.0f ? g : 0.0f) * u;
             } else {
                 h[k] = u > 0.0f ? u : 0.0f;
             }
         }
-        /* y_j = sum over k in ascending order; the k loop is outermost only so
-         * that memory is walked row by row, each y_j still adds k = 0, 1, ... */
-        for (int32_t j = 0; j < d; ++j) acc[j] = 0.0;
-        for (int32_t k = 0; k < K; ++k) {
-            double hk = (double)h[k];
-            const float *row = w_downT_c + (size_t)k * d;
-            for (int32_t j = 0; j < d; ++j) acc[j] += hk * (double)row[j];
+        /* y_j = sum over k in ascending order.  Columns are handed to the threads in
+         * blocks; within a block the k loop is outermost only so that memory is walked
+         * row by row: each y_j still adds k = 0, 1, ... in that order, whatever the
+         * number of threads. */
+#ifdef _OPENMP
+#pragma omp parallel for schedule(static)
+#endif
+        for (int32_t j0 = 0; j0 < d; j0 += 64) {
+            const int32_t j1 = j0 + 64 < d ? j0 + 64 : d;
+            for (int32_t j = j0; j < j1; ++j) acc[j] = 0;
+            for (int32_t k = 0; k < K; ++k) {
+                acc_t hk = (acc_t)h[k];
+                const float *row = w_downT_c + (size_t)k * d;
+                for (int32_t j = j0; j < j1; ++j) acc[j] += hk * (acc_t)row[j];
+            }
+            for (int32_t j = j0; j < j1; ++j)
+                y[(size_t)b * d + j] = (float)(acc[j] + (b_down ? (acc_t)b_down[j] : (acc_t)0));
         }
-        for (int32_t j = 0; j < d; ++j)
-            y[(size_t)b * d + j] = (float)(acc[j] + (b_down ? (double)b_down[j] : 0.0));
         if (h_out) memcpy(h_out + (size_t)b * K, h, sizeof(float) * (size_t)K);
     }
     free(h);

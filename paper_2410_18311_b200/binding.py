@@ -23,7 +23,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = ran
 SYMBOLS = (
     "coreinfer_count", "coreinfer_last_error",
     "coreinfer_select_workspace_bytes", "coreinfer_select_core",
-    "coreinfer_compact",
+    "coreinfer_compact", "coreinfer_verify_core_idx",
     "coreinfer_ffn_decode_workspace_bytes", "coreinfer_ffn_decode",
     "coreinfer_ffn_decode_stack_workspace_bytes", "coreinfer_ffn_decode_stack",
     "coreinfer_ffn_decode_stack_noalloc",
@@ -82,6 +82,8 @@ def load() -> ctypes.CDLL:
     lib.coreinfer_select_core.argtypes = [vp, ctypes.c_int, i32, i32, i64, f64, f64, vp, vp, vp, sz, vp]
     lib.coreinfer_compact.restype = ctypes.c_int
     lib.coreinfer_compact.argtypes = [vp, vp, vp, vp, ctypes.c_int, i32, i32, vp, i32, vp, vp, vp, vp, vp]
+    lib.coreinfer_verify_core_idx.restype = ctypes.c_int
+    lib.coreinfer_verify_core_idx.argtypes = [vp, i32, i32, vp, vp]
     lib.coreinfer_ffn_decode_workspace_bytes.restype = sz
     lib.coreinfer_ffn_decode_workspace_bytes.argtypes = [i32, i32, i32]
     lib.coreinfer_ffn_decode.restype = ctypes.c_int
@@ -159,6 +161,12 @@ def coreinfer_compact(w_up, w_gate, w_down, b_up, core_idx, K, w_up_c, w_gate_c,
     _check(load().coreinfer_compact(_p(w_up), _p(w_gate), _p(w_down), _p(b_up), dtype_code(w_up), d_model,
                                     d_ff, _p(core_idx), int(K), _p(w_up_c), _p(w_gate_c), _p(w_downT_c),
                                     _p(b_up_c), _stream(stream)))
+
+
+def coreinfer_verify_core_idx(core_idx, d_ff, report, stream=None, K=None):
+    """report: CUDA int32 [2] <- (number of bad positions, first bad position or INT32_MAX)."""
+    _check(load().coreinfer_verify_core_idx(_p(core_idx), core_idx.numel() if K is None else int(K), int(d_ff),
+                                            _p(report), _stream(stream)))
 
 
 def coreinfer_ffn_decode_workspace_bytes(batch: int, d_model: int, K: int) -> int:

@@ -60,9 +60,39 @@ gather_cols_T_kernel(const U* __restrict__ w_down, const int32_t* __restrict__ S
     }
 }
 
+// report[0]: number of positions k whose index is out of [0, d_ff) or not above its predecessor;
+// report[1]: the first such position (INT_MAX while there is none).
+__global__ void verify_core_idx_kernel(const int32_t* __restrict__ idx, int K, int d_ff, int32_t* report)
+{
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= K) return;
+    const int32_t v = idx[k];
+    const bool bad = v < 0 || v >= d_ff || (k > 0 && idx[k - 1] >= v);
+    if (bad) {
+        atomicAdd(&report[0], 1);
+        atomicMin(&report[1], k);
+    }
+}
+
 }  // namespace coreinfer
 
 using namespace coreinfer;
+
+extern "C" coreinfer_status coreinfer_verify_core_idx(const int32_t* core_idx, int32_t K, int32_t d_ff,
+                                                      int32_t* report, void* cuda_stream)
+{
+    if (!core_idx || !report) CI_FAIL(COREINFER_ERR_INVALID_ARG, "core_idx / report is NULL");
+    if (d_ff < 1 || K < 1 || K > d_ff) CI_FAIL(COREINFER_ERR_INVALID_ARG, "K = %d outside 1..d_ff (%d)", K, d_ff);
+    DeviceInfo di;
+    coreinfer_status s = device_info(&di);
+    if (s != COREINFER_OK) return s;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    static const int32_t init[2] = {0, 0x7fffffff};
+    CI_CUDA(cudaMemcpyAsync(report, init, sizeof init, cudaMemcpyHostToDevice, st));
+    verify_core_idx_kernel<<<(K + 255) / 256, 256, 0, st>>>(core_idx, K, d_ff, report);
+    CI_CUDA(cudaGetLastError());
+    return COREINFER_OK;
+}
 
 extern "C" coreinfer_status coreinfer_compact(const void* w_up, const void* w_gate, const void* w_down,
                                               const void* b_up, coreinfer_dtype dtype, int32_t d_model,

@@ -4,6 +4,7 @@ import pytest
 import torch
 
 import oracle
+import paper_2410_18311_b200 as ci
 from helpers import require_gpu, gpu_compact, raw_np
 
 pytestmark = pytest.mark.gpu
@@ -32,3 +33,24 @@ def test_compact_bytes(dtype, gated, bias, d, N, K):
         assert raw_np(gate_c).tobytes() == o_gate.tobytes()
     if bias:
         assert raw_np(bup_c).tobytes() == o_bup.tobytes()
+
+
+def test_verify_core_idx_reports_the_first_bad_position():
+    """The index check that guards coreinfer_compact (which trusts its list): a valid list passes,
+    and every kind of defect -- out of range, negative, repeated, descending -- is counted and
+    located.  Only the list itself is read, so bad lists are safe to test."""
+    require_gpu()
+    d_ff = 1000
+    good = torch.arange(0, 900, 3, dtype=torch.int32, device="cuda")
+    report = torch.empty(2, dtype=torch.int32, device="cuda")
+    ci.coreinfer_verify_core_idx(good, d_ff, report)
+    assert report.cpu().tolist() == [0, 2 ** 31 - 1]
+    S_o, _ = oracle.select(np.abs(np.random.default_rng(0).standard_normal((7, d_ff))).astype(np.float32), 0.4, 0.2)
+    ci.coreinfer_verify_core_idx(torch.from_numpy(S_o).cuda(), d_ff, report)      # a set as the oracle emits it
+    assert report.cpu().tolist() == [0, 2 ** 31 - 1]
+    for pos, val, nbad in [(17, 1000, 2), (0, -1, 1), (40, 40 * 3 - 3, 1), (299, 5, 1), (120, 2 ** 31 - 1, 2)]:
+        bad = good.clone()
+        bad[pos] = val
+        ci.coreinfer_verify_core_idx(bad, d_ff, report)
+        n, first = report.cpu().tolist()
+        assert first == pos and n == nbad, (pos, val, n, first)

@@ -185,3 +185,20 @@ def test_glue_closed_forms():
     s = (a.astype(np.float64) + b)
     np.testing.assert_allclose(out, s / np.sqrt(np.mean(s * s)), rtol=1e-6)
     np.testing.assert_allclose(oracle.glue(4 * a, 4 * b), out, rtol=1e-6)    # scale-free
+
+
+def test_fp32_accumulators_stay_close_to_the_double_oracle():
+    """The oracle keeps double running sums (a sequential fp32 sum over thousands of terms would
+    spend part of the 1e-4 budget by itself).  The fp32-accumulator build of the same loops is
+    reported against it: its distance must stay far below the bf16 gate and is printed."""
+    rng = np.random.default_rng(11)
+    d, K = 4096, 700
+    x = rng.standard_normal((2, d)).astype(np.float32)
+    up = (rng.standard_normal((K, d)) * 0.02).astype(np.float32)
+    down = (rng.standard_normal((K, d)) * 0.02).astype(np.float32)
+    y64 = oracle.ffn(x, oracle.RELU, up, None, down)
+    y32 = oracle.ffn_f32_accumulators(x, oracle.RELU, up, None, down)
+    rms = np.sqrt(np.mean(y64.astype(np.float64) ** 2, axis=-1, keepdims=True))
+    dist = float(np.max(np.abs(y32.astype(np.float64) - y64) / rms))
+    print("fp32-accumulator FFN vs double-accumulator oracle: %.3g of the output RMS (d=%d, K=%d)" % (dist, d, K))
+    assert 0.0 < dist < 1e-4
