@@ -419,6 +419,7 @@ struct MmaStackParams {
     __nv_bfloat16* x_layers;      // [L][B][d] or NULL (row 0 is written by the host)
     float* ybuf;                  // [3][B][d]; buffers 0 and 1 zero on entry
     unsigned* ctrl;               // [0] status word, [1] grid-barrier arrivals; zero on entry
+    unsigned long long* stamps;   // [CTA][layer][kStampSlots] cycle counts, or NULL (COREINFER_STAMPS builds)
     StackLayerB layers[COREINFER_MAX_LAYERS];
 };
 
@@ -607,6 +608,7 @@ decode_batch_stack_kernel(const __grid_constant__ MmaStackParams p)
         if (slot >= NS) { slot -= NS; phase ^= 1u; }
     };
     const uint32_t zero_addr = smem_u32(zero_row);
+    unsigned long long* const stamps = tid == 0 ? p.stamps : nullptr;
 
     for (int l = 0; l < p.L; ++l) {
         const StackLayerB& ly = p.layers[l];
@@ -617,6 +619,9 @@ decode_batch_stack_kernel(const __grid_constant__ MmaStackParams p)
         const int n_dn_units = (n + UR - 1) / UR;
         const bool last = (l == p.L - 1);
         float* ytarget = p.y_layers ? p.y_layers + (size_t)l * row : (last ? p.y_last : p.ybuf + (size_t)(l % 3) * row);
+        const size_t sb = ((size_t)cta * p.L + l) * kStampSlots;
+        (void)sb;
+        CI_STAMP(stamps, sb, 0);
 
         // ---------------------------------------------------- up (+ gate) units --
         for (int u = 0; u < n_up_units; ++u) {
@@ -683,6 +688,7 @@ decode_batch_stack_kernel(const __grid_constant__ MmaStackParams p)
             named_bar_sync(1, kMmaThreads);
         }
 
+        CI_STAMP(stamps, sb, 1);
         // ------------------------------------------------------------ down units --
         float dacc[kMmaMaxTiles][4];
 #pragma unroll
@@ -713,6 +719,7 @@ decode_batch_stack_kernel(const __grid_constant__ MmaStackParams p)
             release_items(cnt);
         }
 
+        CI_STAMP(stamps, sb, 3);
         // ---------------------------------------------------------------- flush --
         float* st = scratch + warp * 128;            // [8 sequences][16 columns]
         named_bar_sync(1, kMmaThreads);              // the up phase's last use of the scratch is over
@@ -738,12 +745,14 @@ decode_batch_stack_kernel(const __grid_constant__ MmaStackParams p)
                 __syncwarp();
             }
         }
-        if (last) break;
+        if (last) { CI_STAMP(stamps, sb, 4); break; }
 
         // ------------------------------------------------- cross-CTA sum, glue --
         named_bar_sync(1, kMmaThreads);              // every consumer's reductions precede the arrival
+        CI_STAMP(stamps, sb, 4);
         if (tid == 0 && !*abort_flag) stack_grid_barrier(p.ctrl, (unsigned)(l + 1) * (unsigned)G, abort_flag);
         named_bar_sync(1, kMmaThreads);
+        CI_STAMP(stamps, sb, 7);
         // the target layer l + 2 will add into, if it is one of the rotating buffers: every CTA
         // has read it for the last time before it arrived at the barrier above
         if (!p.y_layers && l + 2 < p.L - 1) {
@@ -775,6 +784,7 @@ decode_batch_stack_kernel(const __grid_constant__ MmaStackParams p)
             ss += __shfl_xor_sync(0xffffffffu, ss, 2);
             if ((lane & 3) == 0) ssq[warp * 8 + nb] = ss;
             named_bar_sync(1, kMmaThreads);
+            CI_STAMP(stamps, sb, 8);
             if (tid == 0) *layers_done = l + 1;      // the sums have been read: the producer may go on
             float tot = 0.f;
 #pragma unroll
@@ -798,6 +808,7 @@ decode_batch_stack_kernel(const __grid_constant__ MmaStackParams p)
                 }
             }
         }
+        CI_STAMP(stamps, sb, 9);
     }
 }
 
@@ -834,6 +845,7 @@ coreinfer_status decode_stack_batched_mma(const coreinfer_layer* layers, int L, 
     p.ybuf = ybuf;
     p.ctrl = ctrl;
     const int G = di.sm_count;
+    p.stamps = stamps_buffer((size_t)G * L * kStampSlots * sizeof(unsigned long long));
     const int rmax = (Kmax + G - 1) / G + 1;
     p.rpad = ((rmax + 15) & ~15) + 16;      // the zeroed tail of h may reach one tile past the slab
     const size_t fixed = mma_fixed_smem(p.slot_stride, p.rpad);
