@@ -493,6 +493,9 @@ def run_ours(args, cfg):
     if not args.no_configs and world == 1:
         del weights, acts, stack
         torch.cuda.empty_cache()
+        pre = prefill_stage_times(ci, wl, cfg, cfg.T, cfg.beta)
+        pre["select_floor_us_at_measured_peak"] = pre["activation_bytes"] / peak / 1e3
+        line["prefill_stage_one_layer"] = pre
         line["configs"] = other_configs(ci, wl, peak, cfg.name)
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = oracle_sample(cfg, n_layers=4, n_tokens=min(cfg.decode_steps, 256))
@@ -545,22 +548,32 @@ def prefill_stage_times(ci, wl, cfg, T, beta, layer=0):
     import torch
     kind = ci.FFN_RELU_GATED if cfg.gated else ci.FFN_RELU
     w_up, w_gate, w_down = wl.layer_weights(cfg, layer, device="cuda")
+    act_us = None
+    stream = torch.cuda.current_stream()
     if cfg.planted:
         A, _ = wl.planted_activations(cfg, layer, T, device="cuda")
     else:
         X = wl.prompt_hidden(cfg, device="cuda", T=T)
         A = torch.empty((T, cfg.d_ff), device="cuda")
-        ci.coreinfer_ffn_dense_ref(X, kind, w_up, w_gate, w_down, None, None, A, None)
+        if cfg.dtype == "bf16":      # the activations as the tensor-core pre-fill produces them
+            tws = torch.empty(ci.coreinfer_prefill_activations_workspace_bytes(), dtype=torch.uint8, device="cuda")
+            act_us = 1e3 * _time_ms(lambda: ci.coreinfer_prefill_activations(X, kind, w_up, w_gate, None, A, tws, stream),
+                                    stream, 10)
+            ci.coreinfer_workspace_status(tws)
+        else:
+            ci.coreinfer_ffn_dense_ref(X, kind, w_up, w_gate, w_down, None, None, A, None)
     K = ci.coreinfer_count(beta, cfg.d_ff)
     S = torch.empty(K, dtype=torch.int32, device="cuda")
     ws = torch.empty(ci.coreinfer_select_workspace_bytes(T, cfg.d_ff), dtype=torch.uint8, device="cuda")
-    stream = torch.cuda.current_stream()
     sel = _time_ms(lambda: ci.coreinfer_select_core(A, cfg.alpha, beta, S, None, ws, stream), stream, 10)
     new = lambda: torch.empty((K, cfg.d_model), dtype=cfg.torch_dtype, device="cuda")
     up_c, down_c, gate_c = new(), new(), (new() if cfg.gated else None)
     cmp_ = _time_ms(lambda: ci.coreinfer_compact(w_up, w_gate, w_down, None, S, K, up_c, gate_c, down_c, None, stream),
                     stream, 5)
-    return {"T": T, "K": K, "select_us": 1e3 * sel, "select_floor_us_at_measured_peak": None,
+    return {"T": T, "K": K, "activations_tensor_core_us": act_us,
+            "activations_tflops": (None if act_us is None else
+                                   2.0 * T * cfg.d_model * cfg.d_ff * (2 if cfg.gated else 1) / act_us / 1e6),
+            "select_us": 1e3 * sel, "select_floor_us_at_measured_peak": None,
             "activation_bytes": 4 * T * cfg.d_ff, "compact_us": 1e3 * cmp_}
 
 

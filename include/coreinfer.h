@@ -274,6 +274,32 @@ coreinfer_status coreinfer_ffn_dense_ref(const void* x, int32_t T, coreinfer_dty
                                          const void* b_up, const void* b_down,
                                          float* h_out, float* y_out, void* cuda_stream);
 
+/* ------------------------------------------------------------------ (5) --
+ * Pre-fill activations on the tensor cores: the [T, d_ff] tensor A that Definition 1 is
+ * applied to, produced the way the method obtains it -- as the intermediate result of the dense
+ * pre-fill pass (Section 4.2, Fig. 1) -- without the down projection:
+ *   RELU:        A = max(X W_up^T + b_up, 0)        RELU_GATED:  A = max(X W_gate^T, 0) * (X W_up^T)
+ * bf16 inputs, exact products, fp32 accumulation (tcgen05.mma into tensor memory), fp32 output.
+ * The summation order differs from coreinfer_ffn_dense_ref's, so the two agree to fp32 rounding
+ * (1e-4 relative), not bit for bit; selection is exact on whichever tensor it is given.
+ *
+ *   x        device [T, d_model] bf16            w_up   device [d_ff, d_model] bf16
+ *   w_gate   device [d_ff, d_model] bf16 or NULL (NULL iff RELU)
+ *   b_up     device [d_ff] bf16 or NULL (RELU only)
+ *   act_out  device out [T, d_ff] fp32 with row stride ld_act elements (ld_act >= d_ff, % 4 == 0)
+ *   workspace  device, at least coreinfer_prefill_activations_workspace_bytes(); its first word is
+ *              a status word readable with coreinfer_workspace_status.
+ * d_model must be a multiple of 8.  Any T and d_ff (edges are zero-filled and masked).
+ * Errors: INVALID_ARG, UNSUPPORTED (fp32 inputs: use coreinfer_ffn_dense_ref), WORKSPACE, CUDA. */
+size_t coreinfer_prefill_activations_workspace_bytes(void);
+
+coreinfer_status coreinfer_prefill_activations(const void* x, int32_t T, coreinfer_dtype dtype,
+                                               coreinfer_ffn_kind kind, int32_t d_model, int32_t d_ff,
+                                               const void* w_up, const void* w_gate, const void* b_up,
+                                               float* act_out, int64_t ld_act,
+                                               void* workspace, size_t workspace_bytes,
+                                               void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

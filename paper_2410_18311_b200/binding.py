@@ -30,6 +30,7 @@ SYMBOLS = (
     "coreinfer_workspace_status",
     "coreinfer_debug_stamps",
     "coreinfer_ffn_dense_ref",
+    "coreinfer_prefill_activations_workspace_bytes", "coreinfer_prefill_activations",
 )
 STAMP_SLOTS = 16
 
@@ -104,6 +105,11 @@ def load() -> ctypes.CDLL:
     lib.coreinfer_ffn_dense_ref.restype = ctypes.c_int
     lib.coreinfer_ffn_dense_ref.argtypes = [vp, i32, ctypes.c_int, ctypes.c_int, i32, i32, vp, vp, vp, vp, vp,
                                             vp, vp, vp]
+    lib.coreinfer_prefill_activations_workspace_bytes.restype = sz
+    lib.coreinfer_prefill_activations_workspace_bytes.argtypes = []
+    lib.coreinfer_prefill_activations.restype = ctypes.c_int
+    lib.coreinfer_prefill_activations.argtypes = [vp, i32, ctypes.c_int, ctypes.c_int, i32, i32, vp, vp, vp, vp, i64,
+                                                  vp, sz, vp]
     _lib = lib
     return lib
 
@@ -238,3 +244,16 @@ def coreinfer_ffn_dense_ref(x, kind, w_up, w_gate, w_down, b_up, b_down, h_out, 
     _check(load().coreinfer_ffn_dense_ref(_p(x), T, dtype_code(x), int(kind), d_model, d_ff, _p(w_up),
                                           _p(w_gate), _p(w_down), _p(b_up), _p(b_down), _p(h_out), _p(y_out),
                                           _stream(stream)))
+
+
+def coreinfer_prefill_activations_workspace_bytes() -> int:
+    return int(load().coreinfer_prefill_activations_workspace_bytes())
+
+
+def coreinfer_prefill_activations(x, kind, w_up, w_gate, b_up, act_out, workspace, stream=None):
+    """x [T, d] bf16, w_up / w_gate [d_ff, d] bf16 -> act_out [T, d_ff] fp32 (tensor cores)."""
+    T, d_model = x.shape
+    d_ff = w_up.shape[0]
+    _check(load().coreinfer_prefill_activations(_p(x), T, dtype_code(x), int(kind), d_model, d_ff, _p(w_up), _p(w_gate),
+                                                _p(b_up), _p(act_out), act_out.stride(0), _p(workspace),
+                                                workspace.numel() * workspace.element_size(), _stream(stream)))
