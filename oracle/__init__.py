@@ -71,6 +71,7 @@ def _load():
 
 RELU = 0
 RELU_GATED = 1
+SILU_GATED = 2      # h = silu(w_gate.x) * (w_up.x); Definition 1 is applied to h unchanged
 
 
 def num_threads() -> int:
@@ -173,7 +174,7 @@ def ffn(x, kind, w_up_c, w_gate_c, w_downT_c, b_up_c=None, b_down=None, return_h
     b_up_c, b_down = _f32(b_up_c), _f32(b_down)
     K = w_up_c.shape[0]
     assert w_up_c.shape == (K, d) and w_downT_c.shape == (K, d)
-    assert (kind == RELU_GATED) == (w_gate_c is not None)
+    assert (kind in (RELU_GATED, SILU_GATED)) == (w_gate_c is not None)
     y = np.empty((B, d), dtype=np.float32)
     h = np.empty((B, max(K, 1)), dtype=np.float32) if return_h else None
     _load().oracle_ffn(_ptr(x), B, int(kind), d, K, _ptr(w_up_c), _ptr(w_gate_c),
@@ -191,7 +192,7 @@ def ffn_dense(x, kind, w_up, w_gate, w_down, b_up=None, b_down=None, want_h=True
     b_up, b_down = _f32(b_up), _f32(b_down)
     N = w_up.shape[0]
     assert w_up.shape == (N, d) and w_down.shape == (d, N)
-    assert (kind == RELU_GATED) == (w_gate is not None)
+    assert (kind in (RELU_GATED, SILU_GATED)) == (w_gate is not None)
     H = np.empty((T, N), dtype=np.float32) if want_h else None
     Y = np.empty((T, d), dtype=np.float32) if want_y else None
     _load().oracle_ffn_dense(_ptr(x), T, int(kind), d, N, _ptr(w_up), _ptr(w_gate),

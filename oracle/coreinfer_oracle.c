@@ -186,9 +186,22 @@ void oracle_compact(const void *w_up, const void *w_gate, const void *w_down,
     }
 }
 
+/* Gate nonlinearity of the gated kinds.  kind 1: ReLU.  kind 2: SiLU, g / (1 + exp(-g)),
+ * the activation of the LLaMA models for which Section 5.1 ("Verification and Analysis") and
+ * the appendix "Generalization to LLaMA3.1-8b" report the same core-neuron behaviour; the
+ * paper gives no separate score for them, so Definition 1 is applied unchanged to the
+ * intermediate h = silu(w_gate.x) * (w_up.x) (entries that are not positive are never core
+ * neurons, as for the ReLU-gated kind).  Evaluated in double, rounded to fp32. */
+static float gate_act(float g, int32_t kind)
+{
+    if (kind == 2) return (float)((double)g / (1.0 + exp(-(double)g)));
+    return g > 0.0f ? g : 0.0f;
+}
+
 /* Decode FFN over compacted weights (Section 4.2: inference through the fixed
- * core neurons only).  kind 0: h = max(w_up.x + b_up, 0); kind 1 (gated):
- * h = max(w_gate.x, 0) * (w_up.x).  y = sum_k h_k * w_downT_c[k] + b_down.
+ * core neurons only).  kind 0: h = max(w_up.x + b_up, 0); kind 1 (ReLU-gated):
+ * h = max(w_gate.x, 0) * (w_up.x); kind 2 (SiLU-gated): h = silu(w_gate.x) * (w_up.x).
+ * y = sum_k h_k * w_downT_c[k] + b_down.
  * x: [B][d]; w_*_c: [K][d]; b_up_c: [K] or NULL; b_down: [d] or NULL;
  * y: [B][d]; h_out: [B][K] or NULL. */
 void oracle_ffn(const float *x, int32_t B, int32_t kind, int32_t d, int32_t K,
@@ -208,12 +221,12 @@ void oracle_ffn(const float *x, int32_t B, int32_t kind, int32_t d, int32_t K,
                 su += (acc_t)w_up_c[(size_t)k * d + i] * (acc_t)xb[i];
             if (kind == 0 && b_up_c) su += (acc_t)b_up_c[k];
             float u = (float)su;
-            if (kind == 1) {
+            if (kind >= 1) {
                 acc_t sg = 0;
                 for (int32_t i = 0; i < d; ++i)
                     sg += (acc_t)w_gate_c[(size_t)k * d + i] * (acc_t)xb[i];
                 float g = (float)sg;
-                h[k] = (g > 0.0f ? g : 0.0f) * u;
+                h[k] = gate_act(g, kind) * u;
             } else {
                 h[k] = u > 0.0f ? u : 0.0f;
             }
@@ -266,12 +279,12 @@ void oracle_ffn_dense(const float *x, int32_t T, int32_t kind, int32_t d, int32_
                     su += (double)w_up[(size_t)n * d + i] * (double)xt[i];
                 if (kind == 0 && b_up) su += (double)b_up[n];
                 float u = (float)su;
-                if (kind == 1) {
+                if (kind >= 1) {
                     double sg = 0.0;
                     for (int32_t i = 0; i < d; ++i)
                         sg += (double)w_gate[(size_t)n * d + i] * (double)xt[i];
                     float g = (float)sg;
-                    h[n] = (g > 0.0f ? g : 0.0f) * u;
+                    h[n] = gate_act(g, kind) * u;
                 } else {
                     h[n] = u > 0.0f ? u : 0.0f;
                 }

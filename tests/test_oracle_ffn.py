@@ -202,3 +202,65 @@ def test_fp32_accumulators_stay_close_to_the_double_oracle():
     dist = float(np.max(np.abs(y32.astype(np.float64) - y64) / rms))
     print("fp32-accumulator FFN vs double-accumulator oracle: %.3g of the output RMS (d=%d, K=%d)" % (dist, d, K))
     assert 0.0 < dist < 1e-4
+
+
+# ---- SiLU-gated kind (h = silu(w_gate.x) * (w_up.x)) --------------------------------------
+def _silu_case(seed=21, B=3, d=96, K=50):
+    rng = np.random.default_rng(seed)
+    x = rng.standard_normal((B, d)).astype(np.float32)
+    up = (rng.standard_normal((K, d)) * 0.3).astype(np.float32)
+    gate = (rng.standard_normal((K, d)) * 0.3).astype(np.float32)
+    down = (rng.standard_normal((K, d)) * 0.3).astype(np.float32)
+    return x, up, gate, down
+
+
+def test_silu_gated_matches_library_sigmoid_and_matmul():
+    """Library routines: float64 matmul and scipy's expit (silu(g) = g * expit(g))."""
+    from scipy.special import expit
+    x, up, gate, down = _silu_case()
+    y, h = oracle.ffn(x, oracle.SILU_GATED, up, gate, down, return_h=True)
+    g = (x.astype(np.float64) @ gate.astype(np.float64).T).astype(np.float32).astype(np.float64)
+    u = (x.astype(np.float64) @ up.astype(np.float64).T).astype(np.float32).astype(np.float64)
+    h_ref = ((g * expit(g)).astype(np.float32).astype(np.float64) * u).astype(np.float32)
+    np.testing.assert_allclose(h, h_ref, rtol=2e-7, atol=1e-30)
+    y_ref = h_ref.astype(np.float64) @ down.astype(np.float64)
+    np.testing.assert_allclose(y, y_ref, rtol=1e-6, atol=1e-6)
+
+
+def test_silu_identities():
+    """silu(a) - silu(-a) = a, silu(0) = 0, silu(a) -> a and silu(-a) -> 0 for large a: a wrong
+    sign or a dropped term breaks one of them.  The layer is built so that h_k = silu(a_k):
+    gate row k picks coordinate k of x, every up row picks the last coordinate (= 1)."""
+    K = 6
+    d = K + 2                                                      # one spare coordinate, d even
+    a = np.array([0.0, 0.5, -1.25, 3.0, 30.0, -30.0], np.float32)
+    gate = np.zeros((K, d), np.float32); gate[np.arange(K), np.arange(K)] = 1.0
+    up = np.zeros((K, d), np.float32); up[:, K] = 1.0
+    down = np.zeros((K, d), np.float32); down[np.arange(K), np.arange(K)] = 1.0
+    x = np.zeros((2, d), np.float32); x[0, :K] = a; x[1, :K] = -a; x[:, K] = 1.0
+    y = oracle.ffn(x, oracle.SILU_GATED, up, gate, down).astype(np.float64)
+    hp, hm = y[0, :K], y[1, :K]
+    np.testing.assert_allclose(hp - hm, a.astype(np.float64), rtol=1e-6, atol=1e-7)
+    assert hp[0] == 0.0 and hm[0] == 0.0
+    np.testing.assert_allclose(hp[4], 30.0, rtol=1e-6)
+    assert abs(hm[4]) < 1e-10 and abs(hp[5]) < 1e-10
+    np.testing.assert_allclose(hp[1], 0.5 / (1.0 + np.exp(-0.5)), rtol=1e-6)   # 0.3112296656...
+    assert abs(hp[1] - 0.31122966560092726) < 1e-7
+
+
+def test_silu_gated_compacted_equals_dense_restricted():
+    x, up, gate, down = _silu_case(seed=5, B=2, d=64, K=40)
+    N = 40
+    w_down = np.ascontiguousarray(down.T)
+    H, Y = oracle.ffn_dense(x, oracle.SILU_GATED, up, gate, w_down)
+    y_all = oracle.ffn(x, oracle.SILU_GATED, up, gate, down)
+    np.testing.assert_array_equal(Y, y_all)                       # same loops over all neurons
+    S = np.array([1, 4, 9, 16, 25, 36], np.int32)
+    y_S = oracle.ffn(x, oracle.SILU_GATED, up[S], gate[S], down[S])
+    mask = np.zeros(N, bool); mask[S] = True
+    y_ref = (np.where(mask, H, 0).astype(np.float64) @ down.astype(np.float64))
+    np.testing.assert_allclose(y_S, y_ref, rtol=1e-6, atol=1e-6)
+    # negative intermediates exist and are never selected by Definition 1
+    assert (H < 0).any()
+    Ssel, f = oracle.select(H, 1.0, 1.0)
+    assert f[(H <= 0).all(axis=0)].sum() == 0
