@@ -50,13 +50,18 @@ typedef enum {
     COREINFER_ERR_TIMEOUT = 5        /* a bounded device-side wait gave up (see coreinfer_workspace_status) */
 } coreinfer_status;
 
-typedef enum { COREINFER_F32 = 0, COREINFER_BF16 = 1 } coreinfer_dtype;
+/* Storage types of weights and layer inputs.  F16 is the type of the paper's runs (Section 5
+ * "Models": FP16 weights, FP32 intermediate activations); the workload configurations use BF16. */
+typedef enum { COREINFER_F32 = 0, COREINFER_BF16 = 1, COREINFER_F16 = 2 } coreinfer_dtype;
 
 /* FFN kinds.  RELU:        h = max(W_up x + b_up, 0)
  *             RELU_GATED:  h = max(W_gate x, 0) * (W_up x)        (no up bias)
- * and in both y = W_down h + b_down.  h is the "activation layer" output A(x)
- * that Definition 1 ranks. */
-typedef enum { COREINFER_FFN_RELU = 0, COREINFER_FFN_RELU_GATED = 1 } coreinfer_ffn_kind;
+ *             SILU_GATED:  h = silu(W_gate x) * (W_up x), silu(g) = g / (1 + exp(-g))   (no up bias)
+ * and in all of them y = W_down h + b_down.  h is the "activation layer" output A(x) that
+ * Definition 1 ranks.  The paper reports core neurons for SiLU models (Section 5.1, appendix
+ * on LLaMA3.1-8b) without giving them another score, so Definition 1 applies to h as it
+ * stands: entries of h that are not positive are never core neurons. */
+typedef enum { COREINFER_FFN_RELU = 0, COREINFER_FFN_RELU_GATED = 1, COREINFER_FFN_SILU_GATED = 2 } coreinfer_ffn_kind;
 
 #define COREINFER_MAX_BATCH 8
 #define COREINFER_MAX_LAYERS 128

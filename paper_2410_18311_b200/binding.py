@@ -14,8 +14,8 @@ import torch
 
 from . import _build
 
-F32, BF16 = 0, 1
-FFN_RELU, FFN_RELU_GATED = 0, 1
+F32, BF16, F16 = 0, 1, 2
+FFN_RELU, FFN_RELU_GATED, FFN_SILU_GATED = 0, 1, 2
 MAX_BATCH, MAX_LAYERS = 8, 128
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
 
@@ -133,6 +133,8 @@ def dtype_code(t: torch.Tensor) -> int:
         return F32
     if t.dtype == torch.bfloat16:
         return BF16
+    if t.dtype == torch.float16:
+        return F16
     raise CoreInferError(ERR_UNSUPPORTED, "unsupported torch dtype %s" % t.dtype)
 
 

@@ -3,6 +3,7 @@
 
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <stdint.h>
 #include <stdio.h>
 #include <stdarg.h>
@@ -30,7 +31,13 @@ void set_error(const char* fmt, ...);
     } while (0)
 
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
-static inline size_t dtype_size(coreinfer_dtype dt) { return dt == COREINFER_BF16 ? 2 : 4; }
+static inline size_t dtype_size(coreinfer_dtype dt) { return dt == COREINFER_F32 ? 4 : 2; }
+static inline bool dtype_known(coreinfer_dtype dt) { return dt == COREINFER_F32 || dt == COREINFER_BF16 || dt == COREINFER_F16; }
+static inline bool kind_known(coreinfer_ffn_kind k)
+{
+    return k == COREINFER_FFN_RELU || k == COREINFER_FFN_RELU_GATED || k == COREINFER_FFN_SILU_GATED;
+}
+static inline bool kind_gated(coreinfer_ffn_kind k) { return k != COREINFER_FFN_RELU; }
 
 // Cached per-device properties (SM count, opt-in shared memory).
 struct DeviceInfo {
@@ -61,6 +68,12 @@ unsigned long long* stamps_buffer(size_t need_bytes);   // NULL unless a large e
 enum : unsigned { kStatusOk = 0u, kStatusTimeout = 5u };
 
 #ifdef __CUDACC__
+
+// Gate nonlinearity of the gated FFN kinds: ReLU, or SiLU g / (1 + exp(-g)) in fp32.
+__device__ __forceinline__ float gate_activation(float g, int silu)
+{
+    return silu ? g / (1.0f + __expf(-g)) : fmaxf(g, 0.f);
+}
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p)
 {

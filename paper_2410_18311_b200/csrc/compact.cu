@@ -100,8 +100,7 @@ extern "C" coreinfer_status coreinfer_compact(const void* w_up, const void* w_ga
                                               void* w_up_c, void* w_gate_c, void* w_downT_c, void* b_up_c,
                                               void* cuda_stream)
 {
-    if (dtype != COREINFER_F32 && dtype != COREINFER_BF16)
-        CI_FAIL(COREINFER_ERR_UNSUPPORTED, "dtype %d is not supported", (int)dtype);
+    if (!dtype_known(dtype)) CI_FAIL(COREINFER_ERR_UNSUPPORTED, "dtype %d is not supported", (int)dtype);
     const size_t es = dtype_size(dtype);
     if (d_model < 1 || d_ff < 1 || ((size_t)d_model * es) % 16 != 0)
         CI_FAIL(COREINFER_ERR_INVALID_ARG, "d_model %d / d_ff %d: a weight row must be a positive multiple of 16 bytes",

@@ -56,6 +56,7 @@ struct DecodeParams {
     int runahead;       // batches of the next layer requested before this layer's exchange is over
     int trickle;        // further batches, requested one by one once this CTA's arrival at the grid barrier is out
     int trickle_gap;    // cycles between two such requests
+    int silu;           // gated FFN: 0 ReLU gate, 1 SiLU gate
     float inv_d;        // 1 / d_model
     int ysum_ofs;       // shared-memory offset of the buffer holding the CTA's partial y
     const void* x0;
@@ -119,6 +120,40 @@ template <> struct Elem<__nv_bfloat16> {
     static __device__ __forceinline__ float load1(const void* p, int i)
     {
         return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[i]);
+    }
+};
+template <> struct Elem<__half> {
+    static constexpr int kPairs = 4;
+    static __device__ __forceinline__ void unpack(const uint4& q, float2 (&f)[4])
+    {
+        const __half2* h = reinterpret_cast<const __half2*>(&q);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) f[c] = __half22float2(h[c]);
+    }
+    // as for bf16: mixed-precision FMA, the fp16 product is exact in fp32, one rounding per add
+    static __device__ __forceinline__ void dot(const uint4& w, const uint4& x, float& a0, float& a1)
+    {
+        const uint32_t ws[4] = {w.x, w.y, w.z, w.w}, xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            asm("{\n\t.reg .b16 wl, wh, xl, xh;\n\t"
+                "mov.b32 {wl, wh}, %2;\n\tmov.b32 {xl, xh}, %3;\n\t"
+                "fma.rn.f32.f16 %0, wl, xl, %0;\n\tfma.rn.f32.f16 %1, wh, xh, %1;\n\t}"
+                : "+f"(a0), "+f"(a1) : "r"(ws[c]), "r"(xs[c]));
+    }
+    static __device__ __forceinline__ uint32_t pack2(float a, float b)
+    {
+        __half2 t = __floats2half2_rn(a, b);
+        return *reinterpret_cast<uint32_t*>(&t);
+    }
+    static __device__ __forceinline__ uint4 pack(const float2 (&f)[4])
+    {
+        return make_uint4(pack2(f[0].x, f[0].y), pack2(f[1].x, f[1].y), pack2(f[2].x, f[2].y),
+                          pack2(f[3].x, f[3].y));
+    }
+    static __device__ __forceinline__ float load1(const void* p, int i)
+    {
+        return __half2float(reinterpret_cast<const __half*>(p)[i]);
     }
 };
 template <> struct Elem<float> {
@@ -501,7 +536,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
                         if (GATED) {
                             float g = 0.f;
                             for (int w = 0; w < nwarps; ++w) g += red[(nwarps + w) * p.rmax + r];
-                            h = fmaxf(g, 0.f) * u;
+                            h = gate_activation(g, p.silu) * u;
                         } else {
                             if (ly.bup) u += E::load1(ly.bup, k0 + r);
                             h = fmaxf(u, 0.f);
@@ -711,10 +746,8 @@ static coreinfer_status launch_shape(int vpt, const DecodeParams& p, int grid, s
 static coreinfer_status check_common(const void* x, int batch, coreinfer_dtype dtype,
                                      coreinfer_ffn_kind kind, int d_model)
 {
-    if (dtype != COREINFER_F32 && dtype != COREINFER_BF16)
-        CI_FAIL(COREINFER_ERR_UNSUPPORTED, "dtype %d is not supported", (int)dtype);
-    if (kind != COREINFER_FFN_RELU && kind != COREINFER_FFN_RELU_GATED)
-        CI_FAIL(COREINFER_ERR_UNSUPPORTED, "ffn kind %d is not supported", (int)kind);
+    if (!dtype_known(dtype)) CI_FAIL(COREINFER_ERR_UNSUPPORTED, "dtype %d is not supported", (int)dtype);
+    if (!kind_known(kind)) CI_FAIL(COREINFER_ERR_UNSUPPORTED, "ffn kind %d is not supported", (int)kind);
     if (batch < 1 || batch > COREINFER_MAX_BATCH)
         CI_FAIL(COREINFER_ERR_UNSUPPORTED, "batch %d outside 1..%d", batch, COREINFER_MAX_BATCH);
     if (d_model < 1 || ((size_t)d_model * dtype_size(dtype)) % 16 != 0)
@@ -725,7 +758,7 @@ static coreinfer_status check_common(const void* x, int batch, coreinfer_dtype d
 
 static coreinfer_status check_layer(const coreinfer_layer& ly, int l, coreinfer_ffn_kind kind)
 {
-    const bool gated = kind == COREINFER_FFN_RELU_GATED;
+    const bool gated = kind_gated(kind);
     if (ly.K < 1) CI_FAIL(COREINFER_ERR_INVALID_ARG, "layer %d: K = %d < 1", l, ly.K);
     if (!ly.w_up_c || !ly.w_downT_c || !aligned16(ly.w_up_c) || !aligned16(ly.w_downT_c))
         CI_FAIL(COREINFER_ERR_INVALID_ARG, "layer %d: w_up_c / w_downT_c NULL or not 16-byte aligned", l);
@@ -755,7 +788,7 @@ static coreinfer_status decode_stack_b1(const coreinfer_layer* layers, int L, co
     if (!workspace || !aligned16(workspace)) CI_FAIL(COREINFER_ERR_WORKSPACE, "workspace is NULL or misaligned");
     if (workspace_bytes < need_ws)
         CI_FAIL(COREINFER_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, need_ws);
-    const bool gated = kind == COREINFER_FFN_RELU_GATED;
+    const bool gated = kind_gated(kind);
     const size_t esize = dtype_size(dtype);
 
     static thread_local DecodeParams p;   // large; filled per call, passed by value to the launch
@@ -782,6 +815,7 @@ static coreinfer_status decode_stack_b1(const coreinfer_layer* layers, int L, co
     if ((unsigned long long)Kmax * (unsigned long long)G >= (1ull << 32))
         CI_FAIL(COREINFER_ERR_UNSUPPORTED, "K = %d is too large for the slab split (K * SM count must stay below 2^32)", Kmax);
     p.inv_d = 1.0f / (float)d_model;
+    p.silu = kind == COREINFER_FFN_SILU_GATED;
     // Consumer threads: every thread owns `vpt` 16-byte vectors of a row; as many warps as the
     // row needs, 16 at most.
     const int vpt = (p.nv + kMaxConsumers - 1) / kMaxConsumers;
@@ -827,6 +861,9 @@ static coreinfer_status decode_stack_b1(const coreinfer_layer* layers, int L, co
     if (dtype == COREINFER_BF16)
         return gated ? launch_shape<__nv_bfloat16, true>(vpt, p, G, smem, st)
                      : launch_shape<__nv_bfloat16, false>(vpt, p, G, smem, st);
+    if (dtype == COREINFER_F16)
+        return gated ? launch_shape<__half, true>(vpt, p, G, smem, st)
+                     : launch_shape<__half, false>(vpt, p, G, smem, st);
     return gated ? launch_shape<float, true>(vpt, p, G, smem, st)
                  : launch_shape<float, false>(vpt, p, G, smem, st);
 }

@@ -30,6 +30,23 @@ template <> struct VecB<__nv_bfloat16> {
         return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[i]);
     }
 };
+template <> struct VecB<__half> {
+    static constexpr int kElems = 8;
+    static __device__ __forceinline__ void unpack(const uint4& q, float (&f)[8])
+    {
+        const __half2* h = reinterpret_cast<const __half2*>(&q);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 t = __half22float2(h[i]);
+            f[2 * i] = t.x;
+            f[2 * i + 1] = t.y;
+        }
+    }
+    static __device__ __forceinline__ float load1(const void* p, int i)
+    {
+        return __half2float(reinterpret_cast<const __half*>(p)[i]);
+    }
+};
 template <> struct VecB<float> {
     static constexpr int kElems = 4;
     static __device__ __forceinline__ void unpack(const uint4& q, float (&f)[4])
@@ -47,7 +64,7 @@ template <typename T, int B, bool GATED>
 __global__ void __launch_bounds__(kUpWarps * 32)
 batch_up_kernel(const uint4* __restrict__ x, const uint4* __restrict__ w_up,
                 const uint4* __restrict__ w_gate, const void* __restrict__ b_up, float* __restrict__ h,
-                int nv, int K)
+                int nv, int K, int silu)
 {
     using V = VecB<T>;
     constexpr int E = V::kElems;
@@ -85,7 +102,7 @@ batch_up_kernel(const uint4* __restrict__ x, const uint4* __restrict__ w_up,
         for (int b = 0; b < B; ++b) {
             float hv;
             if (GATED) {
-                hv = fmaxf(g[b], 0.f) * u[b];
+                hv = gate_activation(g[b], silu) * u[b];
             } else {
                 float t = u[b] + (b_up ? V::load1(b_up, k) : 0.f);
                 hv = fmaxf(t, 0.f);
@@ -138,7 +155,7 @@ batch_down_kernel(const float* __restrict__ h, const uint4* __restrict__ w_down,
 }
 
 template <typename T, int B>
-static coreinfer_status run_b(const void* x, bool gated, int d_model, const coreinfer_layer& ly, float* y,
+static coreinfer_status run_b(const void* x, bool gated, int silu, int d_model, const coreinfer_layer& ly, float* y,
                               float* h, cudaStream_t st)
 {
     const int K = ly.K;
@@ -147,10 +164,10 @@ static coreinfer_status run_b(const void* x, bool gated, int d_model, const core
     const int gu = (K + kUpWarps - 1) / kUpWarps;
     if (gated)
         batch_up_kernel<T, B, true><<<gu, kUpWarps * 32, 0, st>>>(
-            (const uint4*)x, (const uint4*)ly.w_up_c, (const uint4*)ly.w_gate_c, nullptr, h, nv, K);
+            (const uint4*)x, (const uint4*)ly.w_up_c, (const uint4*)ly.w_gate_c, nullptr, h, nv, K, silu);
     else
         batch_up_kernel<T, B, false><<<gu, kUpWarps * 32, 0, st>>>(
-            (const uint4*)x, (const uint4*)ly.w_up_c, nullptr, ly.b_up_c, h, nv, K);
+            (const uint4*)x, (const uint4*)ly.w_up_c, nullptr, ly.b_up_c, h, nv, K, 0);
     CI_CUDA(cudaGetLastError());
     dim3 gd((nv + kDownThreads - 1) / kDownThreads, (K + kDownRows - 1) / kDownRows);
     batch_down_kernel<T, B><<<gd, kDownThreads, 0, st>>>(h, (const uint4*)ly.w_downT_c, ly.b_down, y, nv, K,
@@ -160,27 +177,27 @@ static coreinfer_status run_b(const void* x, bool gated, int d_model, const core
 }
 
 template <typename T>
-static coreinfer_status run_t(int batch, const void* x, bool gated, int d_model, const coreinfer_layer& ly,
+static coreinfer_status run_t(int batch, const void* x, bool gated, int silu, int d_model, const coreinfer_layer& ly,
                               float* y, float* h, cudaStream_t st)
 {
     switch (batch) {
-        case 2: return run_b<T, 2>(x, gated, d_model, ly, y, h, st);
-        case 3: return run_b<T, 3>(x, gated, d_model, ly, y, h, st);
-        case 4: return run_b<T, 4>(x, gated, d_model, ly, y, h, st);
-        case 5: return run_b<T, 5>(x, gated, d_model, ly, y, h, st);
-        case 6: return run_b<T, 6>(x, gated, d_model, ly, y, h, st);
-        case 7: return run_b<T, 7>(x, gated, d_model, ly, y, h, st);
-        case 8: return run_b<T, 8>(x, gated, d_model, ly, y, h, st);
+        case 2: return run_b<T, 2>(x, gated, silu, d_model, ly, y, h, st);
+        case 3: return run_b<T, 3>(x, gated, silu, d_model, ly, y, h, st);
+        case 4: return run_b<T, 4>(x, gated, silu, d_model, ly, y, h, st);
+        case 5: return run_b<T, 5>(x, gated, silu, d_model, ly, y, h, st);
+        case 6: return run_b<T, 6>(x, gated, silu, d_model, ly, y, h, st);
+        case 7: return run_b<T, 7>(x, gated, silu, d_model, ly, y, h, st);
+        case 8: return run_b<T, 8>(x, gated, silu, d_model, ly, y, h, st);
         default: CI_FAIL(COREINFER_ERR_UNSUPPORTED, "batch %d not built", batch);
     }
 }
 
 // decode_batch_mma.cu: tensor-core kernel for bf16 rows of up to 4096 columns
-coreinfer_status decode_batched_mma(const void* x, int batch, bool gated, int d_model, const coreinfer_layer& ly,
+coreinfer_status decode_batched_mma(const void* x, int batch, bool gated, int silu, int d_model, const coreinfer_layer& ly,
                                     float* y, unsigned* status, const DeviceInfo& di, cudaStream_t st);
 bool decode_batched_mma_serves(int d_model, int K, const DeviceInfo& di);
 coreinfer_status decode_stack_batched_mma(const coreinfer_layer* layers, int L, const void* x0, int batch, bool gated,
-                                          int d_model, float* y_last, float* y_layers, void* x_layers, float* ybuf,
+                                          int silu, int d_model, float* y_last, float* y_layers, void* x_layers, float* ybuf,
                                           unsigned* ctrl, const DeviceInfo& di, cudaStream_t st);
 
 coreinfer_status decode_batched(const void* x, int batch, coreinfer_dtype dtype, coreinfer_ffn_kind kind,
@@ -190,23 +207,27 @@ coreinfer_status decode_batched(const void* x, int batch, coreinfer_dtype dtype,
     DeviceInfo di;
     coreinfer_status s = device_info(&di);
     if (s != COREINFER_OK) return s;
-    const bool gated = kind == COREINFER_FFN_RELU_GATED;
+    const bool gated = kind_gated(kind);
+    const int silu = kind == COREINFER_FFN_SILU_GATED;
     if (clear_status) CI_CUDA(cudaMemsetAsync(workspace, 0, kCtrlBytesB, st));   // status word
     if (dtype == COREINFER_BF16) {
-        s = decode_batched_mma(x, batch, gated, d_model, ly, y, (unsigned*)workspace, di, st);
+        s = decode_batched_mma(x, batch, gated, silu, d_model, ly, y, (unsigned*)workspace, di, st);
         if (s != COREINFER_ERR_UNSUPPORTED) return s;          // otherwise: shape not built there, use the plain kernels
     }
     float* h = (float*)((uint8_t*)workspace + kCtrlBytesB);
-    if (dtype == COREINFER_BF16) return run_t<__nv_bfloat16>(batch, x, gated, d_model, ly, y, h, st);
-    return run_t<float>(batch, x, gated, d_model, ly, y, h, st);
+    if (dtype == COREINFER_BF16) return run_t<__nv_bfloat16>(batch, x, gated, silu, d_model, ly, y, h, st);
+    if (dtype == COREINFER_F16) return run_t<__half>(batch, x, gated, silu, d_model, ly, y, h, st);
+    return run_t<float>(batch, x, gated, silu, d_model, ly, y, h, st);
 }
 
 // ------------------------------------------------------------- stack, batch 2..8 --
 static __device__ __forceinline__ float to_f(float v) { return v; }
 static __device__ __forceinline__ float to_f(__nv_bfloat16 v) { return __bfloat162float(v); }
+static __device__ __forceinline__ float to_f(__half v) { return __half2float(v); }
 template <typename T> static __device__ __forceinline__ T from_f(float v);
 template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+template <> __device__ __forceinline__ __half from_f<__half>(float v) { return __float2half_rn(v); }
 
 // Glue between two layers for the per-layer path, one CTA per sequence: x_next = round((x + y) /
 // rms(x + y)), the same formula (rsqrtf of the mean square) as in the batch-1 stack kernel.
@@ -268,7 +289,8 @@ coreinfer_status decode_stack_batched(const coreinfer_layer* layers, int L, cons
     uint8_t* y0 = w + align256(kCtrlBytesB + (size_t)batch * Kmax * sizeof(float));
     float* ybuf = (float*)y0;                                    // three buffers, ybytes apart
     uint8_t* xbuf[2] = {y0 + 3 * ybytes, y0 + 4 * ybytes};
-    const bool gated = kind == COREINFER_FFN_RELU_GATED;
+    const bool gated = kind_gated(kind);
+    const int silu = kind == COREINFER_FFN_SILU_GATED;
 
     DeviceInfo di;
     coreinfer_status s = device_info(&di);
@@ -284,7 +306,7 @@ coreinfer_status decode_stack_batched(const coreinfer_layer* layers, int L, cons
         if (y_layers) CI_CUDA(cudaMemsetAsync(y_layers, 0, (size_t)L * row * sizeof(float), st));
         CI_CUDA(cudaMemsetAsync(y_last, 0, row * sizeof(float), st));
         CI_CUDA(cudaMemsetAsync(ybuf, 0, 2 * ybytes, st));
-        s = decode_stack_batched_mma(layers, L, x0, batch, gated, d_model, y_last, y_layers, x_layers, ybuf,
+        s = decode_stack_batched_mma(layers, L, x0, batch, gated, silu, d_model, y_last, y_layers, x_layers, ybuf,
                                      (unsigned*)workspace, di, st);
         if (s != COREINFER_ERR_UNSUPPORTED) {
             if (s != COREINFER_OK) return s;
@@ -310,6 +332,9 @@ coreinfer_status decode_stack_batched(const coreinfer_layer* layers, int L, cons
         if (dtype == COREINFER_BF16)
             batch_glue_kernel<__nv_bfloat16><<<batch, 256, 0, st>>>((const __nv_bfloat16*)x_in, y_out, (__nv_bfloat16*)x_next,
                                                                    (__nv_bfloat16*)dump, d_model, 1.0f / (float)d_model);
+        else if (dtype == COREINFER_F16)
+            batch_glue_kernel<__half><<<batch, 256, 0, st>>>((const __half*)x_in, y_out, (__half*)x_next, (__half*)dump,
+                                                            d_model, 1.0f / (float)d_model);
         else
             batch_glue_kernel<float><<<batch, 256, 0, st>>>((const float*)x_in, y_out, (float*)x_next, (float*)dump,
                                                            d_model, 1.0f / (float)d_model);

@@ -37,6 +37,7 @@ struct MmaParams {
     float* y;                   // [B][d], zero on entry
     unsigned* status;
     int K, d, B, row_bytes, slot_stride, n_slots, rpad;
+    int silu;                   // gated: 0 ReLU gate, 1 SiLU gate
 };
 
 // shared memory besides the ring: zero row, barriers, scratch, h parts, flags, sums of squares
@@ -257,7 +258,7 @@ decode_batch_mma_kernel(const MmaParams p)
             float h = 0.f;
             if (r < cnt) {
                 if (GATED) {
-                    h = fmaxf(gg, 0.f) * uu;
+                    h = gate_activation(gg, p.silu) * uu;
                 } else {
                     if (p.bup) uu += __bfloat162float(p.bup[k0 + u * RU + r]);
                     h = fmaxf(uu, 0.f);
@@ -338,7 +339,7 @@ decode_batch_mma_kernel(const MmaParams p)
 
 // Returns COREINFER_ERR_UNSUPPORTED (without setting an error text) when the shape is not built here.
 // y is cleared here, on the stream, before the launch.
-coreinfer_status decode_batched_mma(const void* x, int batch, bool gated, int d_model, const coreinfer_layer& ly,
+coreinfer_status decode_batched_mma(const void* x, int batch, bool gated, int silu, int d_model, const coreinfer_layer& ly,
                                     float* y, unsigned* status, const DeviceInfo& di, cudaStream_t st)
 {
     if (d_model % (kMmaWarps * 16) != 0 || d_model / (kMmaWarps * 16) > kMmaMaxTiles) return COREINFER_ERR_UNSUPPORTED;
@@ -351,6 +352,7 @@ coreinfer_status decode_batched_mma(const void* x, int batch, bool gated, int d_
     p.x = (const __nv_bfloat16*)x;
     p.y = y;
     p.status = status;
+    p.silu = silu;
     p.K = ly.K;
     p.d = d_model;
     p.B = batch;
@@ -411,6 +413,7 @@ struct StackLayerB {
 
 struct MmaStackParams {
     int L, d, B, row_bytes, slot_stride, n_slots, rpad;
+    int silu;                     // gated: 0 ReLU gate, 1 SiLU gate
     int runahead;                 // ring items of the next layer the producer may request before this layer's exchange is over
     float inv_d;
     const __nv_bfloat16* x0;      // [B][d]
@@ -663,7 +666,7 @@ decode_batch_stack_kernel(const __grid_constant__ MmaStackParams p)
                 float h = 0.f;
                 if (r < cnt) {
                     if (GATED) {
-                        h = fmaxf(gg, 0.f) * uu;
+                        h = gate_activation(gg, p.silu) * uu;
                     } else {
                         if (ly.bup) uu += __bfloat162float(ly.bup[k0 + u * RU + r]);
                         h = fmaxf(uu, 0.f);
@@ -816,7 +819,7 @@ decode_batch_stack_kernel(const __grid_constant__ MmaStackParams p)
 // checked them (decode_batched_mma_serves), cleared ctrl (256 bytes), y_last, y_layers (when
 // given) and the first two of the three rotating buffers at ybuf.
 coreinfer_status decode_stack_batched_mma(const coreinfer_layer* layers, int L, const void* x0, int batch, bool gated,
-                                          int d_model, float* y_last, float* y_layers, void* x_layers, float* ybuf,
+                                          int silu, int d_model, float* y_last, float* y_layers, void* x_layers, float* ybuf,
                                           unsigned* ctrl, const DeviceInfo& di, cudaStream_t st)
 {
     static thread_local MmaStackParams p;
@@ -832,6 +835,7 @@ coreinfer_status decode_stack_batched_mma(const coreinfer_layer* layers, int L, 
         Kmax = layers[l].K > Kmax ? layers[l].K : Kmax;
     }
     p.L = L;
+    p.silu = silu;
     p.d = d_model;
     p.B = batch;
     p.row_bytes = d_model * 2;

@@ -14,13 +14,14 @@ constexpr int kGemmThreads = 256;
 template <typename T> __device__ __forceinline__ float to_f32(T v);
 template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
 template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <> __device__ __forceinline__ float to_f32<__half>(__half v) { return __half2float(v); }
 
 // C[M, Nn] = epilogue(A[M, Kk] . B[Nn, Kk]^T).  GATED: a second B matrix (the gate) and
 // C = max(A.Bg^T, 0) * (A.B^T); otherwise C = A.B^T + bias[n], with ReLU if RELU.
 template <typename TA, typename TB, bool GATED, bool RELU>
 __global__ void __launch_bounds__(kGemmThreads)
 gemm_nt_kernel(const TA* __restrict__ A, const TB* __restrict__ B, const TB* __restrict__ Bg,
-               const TB* __restrict__ bias, float* __restrict__ C, int M, int Nn, int Kk)
+               const TB* __restrict__ bias, float* __restrict__ C, int M, int Nn, int Kk, int silu)
 {
     __shared__ float As[kBK][kBM + 4];
     __shared__ float Bs[kBK][kBN + 4];
@@ -84,7 +85,7 @@ gemm_nt_kernel(const TA* __restrict__ A, const TB* __restrict__ B, const TB* __r
             if (n >= Nn) continue;
             float v;
             if (GATED) {
-                v = fmaxf(accg[i][j], 0.f) * acc[i][j];
+                v = gate_activation(accg[i][j], silu) * acc[i][j];
             } else {
                 v = acc[i][j] + (bias ? to_f32<TB>(bias[n]) : 0.f);
                 if (RELU) v = fmaxf(v, 0.f);
@@ -95,7 +96,7 @@ gemm_nt_kernel(const TA* __restrict__ A, const TB* __restrict__ B, const TB* __r
 }
 
 template <typename T>
-static coreinfer_status dense_t(const void* x, int T_, bool gated, int d, int N, const void* w_up,
+static coreinfer_status dense_t(const void* x, int T_, bool gated, int silu, int d, int N, const void* w_up,
                                 const void* w_gate, const void* w_down, const void* b_up, const void* b_down,
                                 float* h_out, float* y_out, cudaStream_t st)
 {
@@ -103,16 +104,16 @@ static coreinfer_status dense_t(const void* x, int T_, bool gated, int d, int N,
         dim3 grid((N + kBN - 1) / kBN, (T_ + kBM - 1) / kBM);
         if (gated)
             gemm_nt_kernel<T, T, true, false><<<grid, kGemmThreads, 0, st>>>(
-                (const T*)x, (const T*)w_up, (const T*)w_gate, nullptr, h_out, T_, N, d);
+                (const T*)x, (const T*)w_up, (const T*)w_gate, nullptr, h_out, T_, N, d, silu);
         else
             gemm_nt_kernel<T, T, false, true><<<grid, kGemmThreads, 0, st>>>(
-                (const T*)x, (const T*)w_up, nullptr, (const T*)b_up, h_out, T_, N, d);
+                (const T*)x, (const T*)w_up, nullptr, (const T*)b_up, h_out, T_, N, d, 0);
         CI_CUDA(cudaGetLastError());
     }
     if (y_out) {
         dim3 grid((d + kBN - 1) / kBN, (T_ + kBM - 1) / kBM);
         gemm_nt_kernel<float, T, false, false><<<grid, kGemmThreads, 0, st>>>(
-            h_out, (const T*)w_down, nullptr, (const T*)b_down, y_out, T_, d, N);
+            h_out, (const T*)w_down, nullptr, (const T*)b_down, y_out, T_, d, N, 0);
         CI_CUDA(cudaGetLastError());
     }
     return COREINFER_OK;
@@ -128,11 +129,10 @@ extern "C" coreinfer_status coreinfer_ffn_dense_ref(const void* x, int32_t T, co
                                                     const void* b_up, const void* b_down, float* h_out,
                                                     float* y_out, void* cuda_stream)
 {
-    if (dtype != COREINFER_F32 && dtype != COREINFER_BF16)
-        CI_FAIL(COREINFER_ERR_UNSUPPORTED, "dtype %d is not supported", (int)dtype);
-    if (kind != COREINFER_FFN_RELU && kind != COREINFER_FFN_RELU_GATED)
-        CI_FAIL(COREINFER_ERR_UNSUPPORTED, "ffn kind %d is not supported", (int)kind);
-    const bool gated = kind == COREINFER_FFN_RELU_GATED;
+    if (!dtype_known(dtype)) CI_FAIL(COREINFER_ERR_UNSUPPORTED, "dtype %d is not supported", (int)dtype);
+    if (!kind_known(kind)) CI_FAIL(COREINFER_ERR_UNSUPPORTED, "ffn kind %d is not supported", (int)kind);
+    const bool gated = kind_gated(kind);
+    const int silu = kind == COREINFER_FFN_SILU_GATED;
     if (T < 1 || d_model < 1 || d_ff < 1)
         CI_FAIL(COREINFER_ERR_INVALID_ARG, "T = %d, d_model = %d, d_ff = %d must be >= 1", T, d_model, d_ff);
     if (!x || !w_up || !w_down) CI_FAIL(COREINFER_ERR_INVALID_ARG, "x / w_up / w_down is NULL");
@@ -146,7 +146,9 @@ extern "C" coreinfer_status coreinfer_ffn_dense_ref(const void* x, int32_t T, co
     if (s != COREINFER_OK) return s;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     if (dtype == COREINFER_BF16)
-        return dense_t<__nv_bfloat16>(x, T, gated, d_model, d_ff, w_up, w_gate, w_down, b_up, b_down, h_out,
+        return dense_t<__nv_bfloat16>(x, T, gated, silu, d_model, d_ff, w_up, w_gate, w_down, b_up, b_down, h_out,
                                       y_out, st);
-    return dense_t<float>(x, T, gated, d_model, d_ff, w_up, w_gate, w_down, b_up, b_down, h_out, y_out, st);
+    if (dtype == COREINFER_F16)
+        return dense_t<__half>(x, T, gated, silu, d_model, d_ff, w_up, w_gate, w_down, b_up, b_down, h_out, y_out, st);
+    return dense_t<float>(x, T, gated, silu, d_model, d_ff, w_up, w_gate, w_down, b_up, b_down, h_out, y_out, st);
 }

@@ -1,6 +1,6 @@
 // Pre-fill activations on the tensor cores: A = act(X W_up^T (+ b_up)), or gated
-// A = max(X W_gate^T, 0) * (X W_up^T): the [T, d_ff] tensor that Definition 1 ranks (the paper
-// obtains it as a by-product of the dense pre-fill pass, Section 4.2 / Fig. 1).  bf16 inputs,
+// A = gate(X W_gate^T) * (X W_up^T), gate = ReLU or SiLU: the [T, d_ff] tensor that Definition 1 ranks (the paper
+// obtains it as a by-product of the dense pre-fill pass, Section 4.2 / Fig. 1).  bf16 or fp16 inputs,
 // exact products, fp32 accumulation in tensor memory, fp32 output.
 //
 // One persistent CTA per SM walks 128 x 128 output tiles.  Warp 0 (one lane) feeds a ring of
@@ -30,11 +30,14 @@ constexpr long long kTcWaitCycles = 3000000000LL;
 struct TcParams {
     int T, N, d;
     int gated;
+    int silu;                   // gated: 0 ReLU gate, 1 SiLU gate
+    uint32_t idesc;             // tcgen05 instruction descriptor (operand formats, tile shape)
     int stages;
     int tiles_m, tiles_n;
     long long ld_out;           // row stride of `out`, elements
     float* out;                 // [T][ld_out] fp32
-    const __nv_bfloat16* bias;  // [N] or NULL (not gated)
+    const void* bias;           // [N] in the input type, or NULL (not gated)
+    int f16;                    // inputs are fp16 (else bf16)
     unsigned* status;
 };
 
@@ -126,8 +129,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     constexpr uint32_t STAGE_BYTES = (1 + NB) * kTcTileBytes;
     constexpr uint32_t ACC_COLS = NB * kTcBN;                  // tensor-memory columns of one accumulator set
     constexpr uint32_t TMEM_COLS = 2 * ACC_COLS;               // two sets: 256 or 512 columns
-    // instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, N = 128, M = 128
-    constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTcBN >> 3) << 17) | ((uint32_t)(kTcBM >> 4) << 24);
+    const uint32_t IDESC = p.idesc;
 
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -247,9 +249,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                         for (int e = 0; e < 4; ++e) {
                             float uu = __uint_as_float(u[j + e]);
                             if (GATED) {
-                                v[e] = fmaxf(__uint_as_float(g[j + e]), 0.f) * uu;
+                                v[e] = gate_activation(__uint_as_float(g[j + e]), p.silu) * uu;
                             } else {
-                                if (p.bias && nbase + j + e < p.N) uu += __bfloat162float(p.bias[nbase + j + e]);
+                                if (p.bias && nbase + j + e < p.N)
+                                    uu += p.f16 ? __half2float(reinterpret_cast<const __half*>(p.bias)[nbase + j + e])
+                                                : __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.bias)[nbase + j + e]);
                                 v[e] = fmaxf(uu, 0.f);
                             }
                         }
@@ -304,8 +308,8 @@ static coreinfer_status encode_fn(EncodeTiledFn* out)
     return COREINFER_OK;
 }
 
-// [rows][cols] bf16 row-major, read in boxes of 128 rows x 64 columns with the 128-byte swizzle.
-static coreinfer_status make_map(CUtensorMap* map, const void* base, int rows, int cols)
+// [rows][cols] bf16 or fp16 row-major, read in boxes of 128 rows x 64 columns with the 128-byte swizzle.
+static coreinfer_status make_map(CUtensorMap* map, const void* base, int rows, int cols, bool f16)
 {
     EncodeTiledFn enc;
     coreinfer_status s = encode_fn(&enc);
@@ -314,7 +318,7 @@ static coreinfer_status make_map(CUtensorMap* map, const void* base, int rows, i
     const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
     const cuuint32_t box[2] = {(cuuint32_t)kTcBK, (cuuint32_t)kTcBM};
     const cuuint32_t estr[2] = {1, 1};
-    const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+    const CUresult r = enc(map, f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) CI_FAIL(COREINFER_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
@@ -334,12 +338,12 @@ coreinfer_status coreinfer_prefill_activations(const void* x, int32_t T, coreinf
                                                const void* b_up, float* act_out, int64_t ld_act, void* workspace,
                                                size_t workspace_bytes, void* cuda_stream)
 {
-    if (dtype != COREINFER_BF16)
-        CI_FAIL(COREINFER_ERR_UNSUPPORTED, "the tensor-core pre-fill takes bf16 inputs (dtype %d given); "
+    if (dtype != COREINFER_BF16 && dtype != COREINFER_F16)
+        CI_FAIL(COREINFER_ERR_UNSUPPORTED, "the tensor-core pre-fill takes bf16 or fp16 inputs (dtype %d given); "
                                            "use coreinfer_ffn_dense_ref for fp32", (int)dtype);
-    if (kind != COREINFER_FFN_RELU && kind != COREINFER_FFN_RELU_GATED)
-        CI_FAIL(COREINFER_ERR_UNSUPPORTED, "ffn kind %d is not supported", (int)kind);
-    const bool gated = kind == COREINFER_FFN_RELU_GATED;
+    if (!kind_known(kind)) CI_FAIL(COREINFER_ERR_UNSUPPORTED, "ffn kind %d is not supported", (int)kind);
+    const bool gated = kind_gated(kind);
+    const bool f16 = dtype == COREINFER_F16;
     if (T < 1 || d_model < 1 || d_ff < 1) CI_FAIL(COREINFER_ERR_INVALID_ARG, "T, d_model, d_ff must be >= 1");
     if (d_model % 8 != 0) CI_FAIL(COREINFER_ERR_INVALID_ARG, "d_model %d: a row must be a multiple of 16 bytes", d_model);
     if (!x || !w_up || !act_out || !aligned16(x) || !aligned16(w_up) || !aligned16(act_out))
@@ -358,20 +362,26 @@ coreinfer_status coreinfer_prefill_activations(const void* x, int32_t T, coreinf
     cudaStream_t st = (cudaStream_t)cuda_stream;
 
     CUtensorMap map_x, map_up, map_gate;
-    if ((s = make_map(&map_x, x, T, d_model)) != COREINFER_OK) return s;
-    if ((s = make_map(&map_up, w_up, d_ff, d_model)) != COREINFER_OK) return s;
-    if ((s = make_map(&map_gate, gated ? w_gate : w_up, d_ff, d_model)) != COREINFER_OK) return s;
+    if ((s = make_map(&map_x, x, T, d_model, f16)) != COREINFER_OK) return s;
+    if ((s = make_map(&map_up, w_up, d_ff, d_model, f16)) != COREINFER_OK) return s;
+    if ((s = make_map(&map_gate, gated ? w_gate : w_up, d_ff, d_model, f16)) != COREINFER_OK) return s;
 
     TcParams p;
     p.T = T;
     p.N = d_ff;
     p.d = d_model;
     p.gated = gated ? 1 : 0;
+    p.silu = kind == COREINFER_FFN_SILU_GATED;
+    p.f16 = f16 ? 1 : 0;
+    // instruction descriptor: fp32 accumulate (bit 4), A and B format (bits 7.. and 10..: 0 fp16, 1 bf16; one
+    // instruction takes both operands in the same format), both K-major, N >> 3 at bit 17, M >> 4 at bit 24
+    const uint32_t fmt = f16 ? 0u : 1u;
+    p.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(kTcBN >> 3) << 17) | ((uint32_t)(kTcBM >> 4) << 24);
     p.tiles_m = (T + kTcBM - 1) / kTcBM;
     p.tiles_n = (d_ff + kTcBN - 1) / kTcBN;
     p.ld_out = ld_act;
     p.out = act_out;
-    p.bias = (const __nv_bfloat16*)b_up;
+    p.bias = b_up;
     p.status = (unsigned*)workspace;
     const size_t stage = (size_t)(gated ? 3 : 2) * kTcTileBytes;
     const size_t fixed = 1024 /* alignment slack */ + (2 * kTcMaxStages + 4) * sizeof(uint64_t) + 64;
