@@ -65,6 +65,16 @@ def _load():
             lib.oracle_ffn_dense.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
             lib.oracle_glue.restype = None
             lib.oracle_glue.argtypes = [vp, vp, i32, vp]
+            lib.oracle_top_by_count.restype = None
+            lib.oracle_top_by_count.argtypes = [vp, i32, i32, vp]
+            lib.oracle_counts_add_set.restype = None
+            lib.oracle_counts_add_set.argtypes = [vp, vp, i32]
+            lib.oracle_core_similarity.restype = None
+            lib.oracle_core_similarity.argtypes = [vp, i32, vp, i32, vp]
+            lib.oracle_nearest_centroid.restype = i32
+            lib.oracle_nearest_centroid.argtypes = [vp, i32, i32, vp, vp]
+            lib.oracle_set_delta.restype = i32
+            lib.oracle_set_delta.argtypes = [vp, i32, vp, vp, vp]
             _lib = lib
     return _lib
 
@@ -206,3 +216,57 @@ def glue(x, y) -> np.ndarray:
     out = np.empty_like(x)
     _load().oracle_glue(_ptr(x), _ptr(y), x.shape[0], _ptr(out))
     return out
+
+
+def _i32(a):
+    return np.ascontiguousarray(a, dtype=np.int32)
+
+
+def top_by_count(counts, frac: float) -> np.ndarray:
+    """The ceil(frac * N) neurons with the largest counts (equal counts: lower index first),
+    ascending: Definition 2's rule applied to any count vector (summed token counts of a prompt
+    that arrived in pieces; per-group membership counts of similarity-guided prediction)."""
+    counts = _i32(counts)
+    N = counts.shape[0]
+    K = count(frac, N)
+    S = np.empty(max(K, 1), dtype=np.int32)
+    _load().oracle_top_by_count(_ptr(counts), N, K, _ptr(S))
+    return S[:K].copy()
+
+
+def group_counts(sets, N: int) -> np.ndarray:
+    """counts[n] = number of the given core sets that hold neuron n (Section 4.1, similarity-guided)."""
+    c = np.zeros(N, dtype=np.int32)
+    for S in sets:
+        S = _i32(S)
+        _load().oracle_counts_add_set(_ptr(c), _ptr(S), S.shape[0])
+    return c
+
+
+def core_similarity(A, B):
+    """(shared, involved) = (|A and B|, |A or B|); Insight-2's similarity is shared / involved."""
+    A, B = _i32(A), _i32(B)
+    out = np.zeros(2, dtype=np.int32)
+    _load().oracle_core_similarity(_ptr(A), A.shape[0], _ptr(B), B.shape[0], _ptr(out))
+    return int(out[0]), int(out[1])
+
+
+def nearest_centroid(centroids, v):
+    """(group, squared distances in double) of the centroid nearest to v; ties go to the lower group."""
+    centroids, v = _f32(centroids), _f32(v).reshape(-1)
+    G, D = centroids.shape
+    d2 = np.empty(G, dtype=np.float64)
+    g = _load().oracle_nearest_centroid(_ptr(centroids), G, D, _ptr(v), _ptr(d2))
+    return int(g), d2
+
+
+def set_delta(slot_neuron, S_new):
+    """Rows to rewrite when the deployed set changes to S_new: (slots, neurons, new slot_neuron)."""
+    slot_neuron = _i32(slot_neuron).copy()
+    S_new = _i32(S_new)
+    K = slot_neuron.shape[0]
+    assert S_new.shape[0] == K
+    slots = np.empty(max(K, 1), dtype=np.int32)
+    neurons = np.empty(max(K, 1), dtype=np.int32)
+    n = _load().oracle_set_delta(_ptr(slot_neuron), K, _ptr(S_new), _ptr(slots), _ptr(neurons))
+    return slots[:n].copy(), neurons[:n].copy(), slot_neuron

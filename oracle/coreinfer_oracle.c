@@ -320,3 +320,84 @@ void oracle_glue(const float *x, const float *y, int32_t d, float *out)
     for (int32_t i = 0; i < d; ++i)
         out[i] = (float)(((double)x[i] + (double)y[i]) / r);
 }
+
+/* ---- core sets over several sentences (Section 3.2 Insight-1/2, Section 4.1) -------------
+ *
+ * The neurons "that appear most frequently": the `K` entries of counts[0..N) with the largest
+ * count, equal counts ordered by lower index, written in ascending index (the same rule as
+ * Definition 2 / Eq. 2 applies to the counts of Eq. 3).  It serves two purposes:
+ *   - the sentence-wise set of a prompt that arrives in pieces: Eq. 3 is a sum over tokens, so
+ *     the counts of the pieces add up and the set of the whole prompt follows from the sum;
+ *   - similarity-guided prediction (Section 4.1): counts[n] = number of sentences of a semantic
+ *     group whose core set holds n, K = ceil(gamma * N). */
+void oracle_top_by_count(const int32_t *counts, int32_t N, int32_t K, int32_t *S)
+{
+    entry_t *ord = (entry_t *)malloc(sizeof(entry_t) * (size_t)(N > 0 ? N : 1));
+    for (int32_t n = 0; n < N; ++n) { ord[n].key = (uint32_t)counts[n]; ord[n].idx = n; }
+    qsort(ord, (size_t)N, sizeof(entry_t), cmp_entry_desc);   /* full sort */
+    for (int32_t i = 0; i < K; ++i) S[i] = ord[i].idx;
+    qsort(S, (size_t)K, sizeof(int32_t), cmp_i32_asc);
+    free(ord);
+}
+
+/* counts[n] += 1 for every member of a core set (one sentence of a semantic group). */
+void oracle_counts_add_set(int32_t *counts, const int32_t *S, int32_t K)
+{
+    for (int32_t i = 0; i < K; ++i) counts[S[i]] += 1;
+}
+
+/* Core-neuron similarity of two sets (Insight-2: "the ratio of identical neurons to the total
+ * number of neurons involved"): out[0] = |A and B|, out[1] = |A or B|.  Quadratic on purpose. */
+void oracle_core_similarity(const int32_t *A, int32_t KA, const int32_t *B, int32_t KB, int32_t *out)
+{
+    int32_t shared = 0;
+    for (int32_t i = 0; i < KA; ++i)
+        for (int32_t j = 0; j < KB; ++j)
+            if (A[i] == B[j]) { ++shared; break; }
+    out[0] = shared;
+    out[1] = KA + KB - shared;
+}
+
+/* Nearest centroid (similarity-guided prediction: the group of an input is the cluster its
+ * feature vector falls into; K-Means assigns a point to the centroid at the smallest Euclidean
+ * distance).  centroids: [G][D]; equal distances go to the lower group.  Squared distances in
+ * double; dist2 (may be NULL) receives them. */
+int32_t oracle_nearest_centroid(const float *centroids, int32_t G, int32_t D, const float *v, double *dist2)
+{
+    int32_t best = 0;
+    double best_d = 0.0;
+    for (int32_t g = 0; g < G; ++g) {
+        double s = 0.0;
+        for (int32_t i = 0; i < D; ++i) {
+            double t = (double)v[i] - (double)centroids[(size_t)g * D + i];
+            s += t * t;
+        }
+        if (dist2) dist2[g] = s;
+        if (g == 0 || s < best_d) { best = g; best_d = s; }
+    }
+    return best;
+}
+
+/* Updating a deployed set in place (Fig. 1: the set may be updated after the stability
+ * estimate; the paper gives no rule, this is the mechanism).  slot_neuron[K] says which neuron
+ * each row of the compacted buffers holds (any order).  Rows whose neuron is not in S_new
+ * (ascending) are reassigned, in ascending slot order, to the members of S_new not held yet, in
+ * ascending neuron order.  Writes the changed (slot, neuron) pairs and updates slot_neuron;
+ * returns their number. */
+int32_t oracle_set_delta(int32_t *slot_neuron, int32_t K, const int32_t *S_new, int32_t *slots, int32_t *neurons)
+{
+    int32_t n_leave = 0, n_enter = 0;
+    for (int32_t p = 0; p < K; ++p) {
+        int keep = 0;
+        for (int32_t j = 0; j < K; ++j) if (S_new[j] == slot_neuron[p]) { keep = 1; break; }
+        if (!keep) slots[n_leave++] = p;
+    }
+    for (int32_t j = 0; j < K; ++j) {
+        int held = 0;
+        for (int32_t p = 0; p < K; ++p) if (slot_neuron[p] == S_new[j]) { held = 1; break; }
+        if (!held) neurons[n_enter++] = S_new[j];
+    }
+    /* both lists have the same length because both sets have K distinct members */
+    for (int32_t i = 0; i < n_leave; ++i) slot_neuron[slots[i]] = neurons[i];
+    return n_leave;
+}
