@@ -279,6 +279,73 @@ coreinfer_status coreinfer_ffn_dense_ref(const void* x, int32_t T, coreinfer_dty
                                          const void* b_up, const void* b_down,
                                          float* h_out, float* y_out, void* cuda_stream);
 
+/* ------------------------------------------------------------------ (6) --
+ * Core sets over several sentences.
+ *
+ * Eq. 3 is a sum over tokens, so the counts of a prompt that arrives in pieces add up, and
+ * similarity-guided prediction (Section 4.1) takes, for a semantic group of training sentences,
+ * "the top gamma neurons that appear most frequently within that semantic group": the count of a
+ * neuron is the number of the group's sentences whose sentence-wise core set holds it.  Both end
+ * in the same rule as Definition 2: the top fraction by count, equal counts to the lower index.
+ *
+ *   coreinfer_counts_add      counts[n] += f[n]                 (f: the counts_out of a piece)
+ *   coreinfer_counts_add_set  counts[core_idx[k]] += 1          (one sentence of a group)
+ *   coreinfer_top_by_count    core_idx <- the coreinfer_count(frac, d_ff) neurons with the largest
+ *                             counts, ascending.  Counts must lie in [0, max_count] (the number
+ *                             of tokens or sentences counted); values outside are clamped.
+ * All pointers device; int32 counts [d_ff]; members of a set must be distinct.
+ * Errors: INVALID_ARG, UNSUPPORTED (d_ff too large for the kernel's shared memory), CUDA. */
+coreinfer_status coreinfer_counts_add(int32_t* counts, const int32_t* f, int32_t d_ff, void* cuda_stream);
+coreinfer_status coreinfer_counts_add_set(int32_t* counts, const int32_t* core_idx, int32_t K, int32_t d_ff,
+                                          void* cuda_stream);
+coreinfer_status coreinfer_top_by_count(const int32_t* counts, int32_t d_ff, int32_t max_count, double frac,
+                                        int32_t* core_idx, void* cuda_stream);
+
+/* Core-neuron similarity of two sets (Section 3.2, Insight-2: "the ratio of identical neurons to
+ * the total number of neurons involved"; the quantity Insight-1 tracks while a sentence grows).
+ * set_a must be ascending, set_b may be in any order; both device.  Writes
+ * shared_involved[0] = |A and B|, shared_involved[1] = |A or B| (device, two int32); the
+ * similarity is their quotient.  Errors: INVALID_ARG, CUDA. */
+coreinfer_status coreinfer_core_similarity(const int32_t* set_a, int32_t K_a, const int32_t* set_b, int32_t K_b,
+                                           int32_t* shared_involved, void* cuda_stream);
+
+/* The semantic group of an input (similarity-guided prediction; appendix on its clustering: K-Means
+ * on a layer's activation): the centroid at the smallest Euclidean distance from the feature
+ * vector v; equal distances go to the lower group.  Which vector represents an input, and the
+ * clustering that produced the centroids, are the caller's.
+ *   centroids device [G, D] fp32; v device [D] fp32; group_out device int32;
+ *   workspace device, 8-byte aligned, at least coreinfer_nearest_centroid_workspace_bytes(G): on
+ *   return it holds the G squared distances as doubles.
+ * Errors: INVALID_ARG, WORKSPACE, CUDA. */
+size_t coreinfer_nearest_centroid_workspace_bytes(int32_t G);
+coreinfer_status coreinfer_nearest_centroid(const float* centroids, int32_t G, int32_t D, const float* v,
+                                            int32_t* group_out, void* workspace, size_t workspace_bytes,
+                                            void* cuda_stream);
+
+/* Changing a deployed core set in place.  Fig. 1 lets the sentence-wise set be updated after a
+ * stability estimate; the paper gives no rule for it.  This call is the mechanism (the estimate
+ * is coreinfer_core_similarity between the deployed and the newly selected set; when to act on
+ * it is the caller's): only the rows whose neuron leaves the set are rewritten.
+ *   slot_neuron   device in/out [K]: the neuron each row of the compacted buffers holds now (any
+ *                 order; after coreinfer_compact it is the core_idx given there).
+ *   core_idx_new  device [K] ascending: the set to deploy.
+ * Rows whose neuron is not in core_idx_new are refilled, in ascending row order, with the
+ * members of core_idx_new not held yet, in ascending neuron order (weights gathered from the
+ * dense matrices as in coreinfer_compact); slot_neuron is updated; n_changed_out (device int32)
+ * receives the number of rows rewritten.  Afterwards the buffers hold exactly the rows of
+ * core_idx_new, in slot_neuron's order, which the decode entry points accept as they are (the
+ * FFN sums over the rows in any order).
+ *   workspace  device, at least coreinfer_update_core_set_workspace_bytes(d_ff, K).
+ * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA. */
+size_t coreinfer_update_core_set_workspace_bytes(int32_t d_ff, int32_t K);
+coreinfer_status coreinfer_update_core_set(const void* w_up, const void* w_gate, const void* w_down,
+                                           const void* b_up, coreinfer_dtype dtype,
+                                           int32_t d_model, int32_t d_ff,
+                                           int32_t* slot_neuron, const int32_t* core_idx_new, int32_t K,
+                                           void* w_up_c, void* w_gate_c, void* w_downT_c, void* b_up_c,
+                                           int32_t* n_changed_out,
+                                           void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* ------------------------------------------------------------------ (5) --
  * Pre-fill activations on the tensor cores: the [T, d_ff] tensor A that Definition 1 is
  * applied to, produced the way the method obtains it -- as the intermediate result of the dense

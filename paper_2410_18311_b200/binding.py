@@ -31,6 +31,9 @@ SYMBOLS = (
     "coreinfer_debug_stamps",
     "coreinfer_ffn_dense_ref",
     "coreinfer_prefill_activations_workspace_bytes", "coreinfer_prefill_activations",
+    "coreinfer_counts_add", "coreinfer_counts_add_set", "coreinfer_top_by_count", "coreinfer_core_similarity",
+    "coreinfer_nearest_centroid_workspace_bytes", "coreinfer_nearest_centroid",
+    "coreinfer_update_core_set_workspace_bytes", "coreinfer_update_core_set",
 )
 STAMP_SLOTS = 16
 
@@ -110,6 +113,23 @@ def load() -> ctypes.CDLL:
     lib.coreinfer_prefill_activations.restype = ctypes.c_int
     lib.coreinfer_prefill_activations.argtypes = [vp, i32, ctypes.c_int, ctypes.c_int, i32, i32, vp, vp, vp, vp, i64,
                                                   vp, sz, vp]
+    lib.coreinfer_counts_add.restype = ctypes.c_int
+    lib.coreinfer_counts_add.argtypes = [vp, vp, i32, vp]
+    lib.coreinfer_counts_add_set.restype = ctypes.c_int
+    lib.coreinfer_counts_add_set.argtypes = [vp, vp, i32, i32, vp]
+    lib.coreinfer_top_by_count.restype = ctypes.c_int
+    lib.coreinfer_top_by_count.argtypes = [vp, i32, i32, f64, vp, vp]
+    lib.coreinfer_core_similarity.restype = ctypes.c_int
+    lib.coreinfer_core_similarity.argtypes = [vp, i32, vp, i32, vp, vp]
+    lib.coreinfer_nearest_centroid_workspace_bytes.restype = sz
+    lib.coreinfer_nearest_centroid_workspace_bytes.argtypes = [i32]
+    lib.coreinfer_nearest_centroid.restype = ctypes.c_int
+    lib.coreinfer_nearest_centroid.argtypes = [vp, i32, i32, vp, vp, vp, sz, vp]
+    lib.coreinfer_update_core_set_workspace_bytes.restype = sz
+    lib.coreinfer_update_core_set_workspace_bytes.argtypes = [i32, i32]
+    lib.coreinfer_update_core_set.restype = ctypes.c_int
+    lib.coreinfer_update_core_set.argtypes = [vp, vp, vp, vp, ctypes.c_int, i32, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp,
+                                              sz, vp]
     _lib = lib
     return lib
 
@@ -259,3 +279,45 @@ def coreinfer_prefill_activations(x, kind, w_up, w_gate, b_up, act_out, workspac
     _check(load().coreinfer_prefill_activations(_p(x), T, dtype_code(x), int(kind), d_model, d_ff, _p(w_up), _p(w_gate),
                                                 _p(b_up), _p(act_out), act_out.stride(0), _p(workspace),
                                                 workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def coreinfer_counts_add(counts, f, stream=None):
+    _check(load().coreinfer_counts_add(_p(counts), _p(f), counts.numel(), _stream(stream)))
+
+
+def coreinfer_counts_add_set(counts, core_idx, stream=None):
+    _check(load().coreinfer_counts_add_set(_p(counts), _p(core_idx), core_idx.numel(), counts.numel(), _stream(stream)))
+
+
+def coreinfer_top_by_count(counts, max_count, frac, core_idx, stream=None):
+    _check(load().coreinfer_top_by_count(_p(counts), counts.numel(), int(max_count), float(frac), _p(core_idx),
+                                         _stream(stream)))
+
+
+def coreinfer_core_similarity(set_a, set_b, shared_involved, stream=None):
+    """set_a ascending; shared_involved: CUDA int32 [2] <- (|A and B|, |A or B|)."""
+    _check(load().coreinfer_core_similarity(_p(set_a), set_a.numel(), _p(set_b), set_b.numel(), _p(shared_involved),
+                                            _stream(stream)))
+
+
+def coreinfer_nearest_centroid_workspace_bytes(G: int) -> int:
+    return int(load().coreinfer_nearest_centroid_workspace_bytes(G))
+
+
+def coreinfer_nearest_centroid(centroids, v, group_out, workspace, stream=None):
+    G, D = centroids.shape
+    _check(load().coreinfer_nearest_centroid(_p(centroids), G, D, _p(v), _p(group_out), _p(workspace),
+                                             workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def coreinfer_update_core_set_workspace_bytes(d_ff: int, K: int) -> int:
+    return int(load().coreinfer_update_core_set_workspace_bytes(d_ff, K))
+
+
+def coreinfer_update_core_set(w_up, w_gate, w_down, b_up, slot_neuron, core_idx_new, w_up_c, w_gate_c, w_downT_c, b_up_c,
+                              n_changed_out, workspace, stream=None):
+    d_ff, d_model = w_up.shape
+    _check(load().coreinfer_update_core_set(_p(w_up), _p(w_gate), _p(w_down), _p(b_up), dtype_code(w_up), d_model, d_ff,
+                                            _p(slot_neuron), _p(core_idx_new), slot_neuron.numel(), _p(w_up_c),
+                                            _p(w_gate_c), _p(w_downT_c), _p(b_up_c), _p(n_changed_out), _p(workspace),
+                                            workspace.numel() * workspace.element_size(), _stream(stream)))

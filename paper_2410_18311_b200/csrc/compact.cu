@@ -60,6 +60,12 @@ gather_cols_T_kernel(const U* __restrict__ w_down, const int32_t* __restrict__ S
     }
 }
 
+__global__ void verify_init_kernel(int32_t* report)
+{
+    report[0] = 0;
+    report[1] = 0x7fffffff;
+}
+
 // report[0]: number of positions k whose index is out of [0, d_ff) or not above its predecessor;
 // report[1]: the first such position (INT_MAX while there is none).
 __global__ void verify_core_idx_kernel(const int32_t* __restrict__ idx, int K, int d_ff, int32_t* report)
@@ -87,8 +93,8 @@ extern "C" coreinfer_status coreinfer_verify_core_idx(const int32_t* core_idx, i
     coreinfer_status s = device_info(&di);
     if (s != COREINFER_OK) return s;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    static const int32_t init[2] = {0, 0x7fffffff};
-    CI_CUDA(cudaMemcpyAsync(report, init, sizeof init, cudaMemcpyHostToDevice, st));
+    verify_init_kernel<<<1, 1, 0, st>>>(report);
+    CI_CUDA(cudaGetLastError());
     verify_core_idx_kernel<<<(K + 255) / 256, 256, 0, st>>>(core_idx, K, d_ff, report);
     CI_CUDA(cudaGetLastError());
     return COREINFER_OK;

@@ -577,7 +577,7 @@ select_top_kernel(const int32_t* __restrict__ f, int N, int K, int T, int32_t* _
     SelShared* sh = reinterpret_cast<SelShared*>(hist + kSelBins);
     int* whist = reinterpret_cast<int*>(sh + 1);                          // [kSelWarps][wstride]
     const int tid = threadIdx.x;
-    for (int i = tid; i < N; i += kSelThreads) fs[at(i)] = f[i];
+    for (int i = tid; i < N; i += kSelThreads) fs[at(i)] = min(max(f[i], 0), T);   // counts lie in [0, T]; anything else is clamped
     const int C = (N + kSelThreads - 1) / kSelThreads;
     const int n0 = min(tid * C, N), n1 = min(n0 + C, N);
 
@@ -671,6 +671,27 @@ static coreinfer_status launch_rows_fast(int grid, size_t smem, cudaStream_t st,
     return COREINFER_OK;
 }
 
+// The K entries of f[0 .. N) with the largest count (all counts in [0, max_count]), ascending.
+coreinfer_status launch_select_top(const int32_t* f, int N, int K, int max_count, int32_t* S, const DeviceInfo& di,
+                                   cudaStream_t st)
+{
+    const int n4 = (N + 3) & ~3;
+    size_t smem_top = ((size_t)n4 + n4 / 32 + 8) * sizeof(int) + kSelBins * sizeof(int) + sizeof(SelShared) + 16;
+    int top_shift = 0;
+    while ((max_count >> top_shift) >= kSelBins) ++top_shift;
+    int wstride = (((max_count >> top_shift) + 1 + 31) & ~31) + 1;   // odd: the warps' copies of a bin fall into different banks
+    if (smem_top + (size_t)kSelWarps * wstride * sizeof(int) <= (size_t)di.smem_optin)
+        smem_top += (size_t)kSelWarps * wstride * sizeof(int);
+    else
+        wstride = 0;
+    if (smem_top > (size_t)di.smem_optin)
+        CI_FAIL(COREINFER_ERR_UNSUPPORTED, "d_ff = %d: the counts do not fit in shared memory", N);
+    CI_CUDA(cudaFuncSetAttribute(select_top_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_top));
+    select_top_kernel<<<1, kSelThreads, smem_top, st>>>(f, N, K, max_count, S, wstride);
+    CI_CUDA(cudaGetLastError());
+    return COREINFER_OK;
+}
+
 }  // namespace coreinfer
 
 using namespace coreinfer;
@@ -754,18 +775,7 @@ coreinfer_status coreinfer_select_core(const void* act, coreinfer_dtype act_dtyp
     select_count_kernel<<<(n4 / 4 + kCountCols - 1) / kCountCols, kCountCols * kCountSlices, 0, st>>>(partial, G, n4, d_ff, f);
     CI_CUDA(cudaGetLastError());
 
-    size_t smem_top = ((size_t)n4 + n4 / 32 + 8) * sizeof(int) + kSelBins * sizeof(int) + sizeof(SelShared) + 16;
-    int top_shift = 0;
-    while ((T >> top_shift) >= kSelBins) ++top_shift;
-    int wstride = (((T >> top_shift) + 1 + 31) & ~31) + 1;        // odd: the warps' copies of a bin fall into different banks
-    if (smem_top + (size_t)kSelWarps * wstride * sizeof(int) <= (size_t)di.smem_optin)
-        smem_top += (size_t)kSelWarps * wstride * sizeof(int);
-    else
-        wstride = 0;
-    CI_CUDA(cudaFuncSetAttribute(select_top_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_top));
-    select_top_kernel<<<1, kSelThreads, smem_top, st>>>(f, d_ff, K, T, core_idx, wstride);
-    CI_CUDA(cudaGetLastError());
-    return COREINFER_OK;
+    return launch_select_top(f, d_ff, K, T, core_idx, di, st);
 }
 
 }  // extern "C"
