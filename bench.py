@@ -29,7 +29,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode_stack_kernel launch at the bench
 # workload, from an ncu capture of a 4-layer launch of the same shapes scaled by the layer count
 # (every layer streams its own weights).  None whenever the kernel has changed since the capture.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"opt6.7b": None}
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"opt6.7b": 219.59e6 / 4 * 32}
 
 
 def parse_args():
@@ -49,6 +49,9 @@ def parse_args():
     ap.add_argument("--decode-only", type=int, default=0, metavar="LAYERS",
                     help="profiling target: only decode launches through the first LAYERS layers of the config "
                          "on random compacted weights (small enough for an ncu capture); prints a short JSON line")
+    ap.add_argument("--prefill-only", type=int, default=0, metavar="LAYERS",
+                    help="profiling target: tensor-core activations, selection and compaction of the first LAYERS "
+                         "layers of the config, nothing else (small enough for an ncu capture); prints a short JSON line")
     ap.add_argument("--tokens", type=int, default=2, help="decode launches per step in --decode-only mode")
     ap.add_argument("--batch", type=int, default=1, help="sequences per decode step in --decode-only mode (1..8)")
     ap.add_argument("--stamps", action="store_true",
@@ -194,11 +197,22 @@ def oracle_sample(cfg, n_layers=2, n_tokens=4, seed_layer=0):
     }
 
 
+def config_dict(cfg, K):
+    """The workload description both arms print."""
+    nbytes = cfg.L * cfg.n_mat * K * cfg.d_model * cfg.esize + cfg.L * 2 * cfg.d_model * 4
+    return {"workload": cfg.name, "L": cfg.L, "d_model": cfg.d_model, "d_ff": cfg.d_ff, "T": cfg.T,
+            "alpha": cfg.alpha, "beta": cfg.beta, "K": K, "decode_steps": cfg.decode_steps, "batch": 1,
+            "gated": cfg.gated, "step": "selection + compaction of all layers, then decode_steps tokens",
+            "l2": "inputs larger than L2 (%.2f GB of compacted weights per token)" % (nbytes / 1e9),
+            "parallelism": "independent requests per GPU, no collective"}
+
+
 def run_reference(args, cfg):
     """--impl reference: the oracle on host cores; each step is one bounded sample."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
+    from oracle import count as oracle_count
     for _ in range(min(args.warmup, 1)):
         oracle_sample(cfg, n_layers=1, n_tokens=1)
     vals, t0 = [], time.perf_counter()
@@ -212,8 +226,7 @@ def run_reference(args, cfg):
         "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * cfg.decode_steps / v, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
-        "config": {"workload": cfg.name, "L": cfg.L, "d_model": cfg.d_model, "d_ff": cfg.d_ff, "T": cfg.T,
-                   "alpha": cfg.alpha, "beta": cfg.beta, "decode_steps": cfg.decode_steps, "batch": 1},
+        "config": config_dict(cfg, oracle_count(cfg.beta, cfg.d_ff)),
         "cpu_baseline": {"value": v, "unit": UNIT, "cores": last["cores"], "kind": "oracle", "sample": last["sample"]},
         "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0, "wall_s": wall,
@@ -469,13 +482,9 @@ def run_ours(args, cfg):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": total_ms_max / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
-        "config": {"workload": cfg.name, "L": cfg.L, "d_model": cfg.d_model, "d_ff": cfg.d_ff, "T": cfg.T,
-                   "alpha": cfg.alpha, "beta": cfg.beta, "K": stack.K, "decode_steps": steps_tok, "batch": 1,
-                   "gated": cfg.gated, "step": "selection + compaction of all layers, then decode_steps tokens",
-                   "l2": "inputs larger than L2 (%.2f GB of compacted weights per token)" % (bytes_tok / 1e9),
-                   "parallelism": "independent requests per GPU, no collective",
-                   "launch": "two CUDA graphs per request (pre-fill stage, decode stage)" if graphs is not None
-                             else "one host call per kernel group"},
+        "config": config_dict(cfg, stack.K),
+        "launch_mode": "two CUDA graphs per request (pre-fill stage, decode stage)" if graphs is not None
+                       else "one host call per kernel group",
         "decode": {"tok_s": steps_tok / (decode_ms * 1e-3), "ms_per_token": decode_ms / steps_tok,
                    "gbs": achieved, "frac_of_8TBs": achieved / 8000.0},
         "select_ms_per_layer": sel_ms, "compact_ms_per_layer": cmp_ms, "prefill_ms_per_request": prefill_ms,
@@ -691,10 +700,65 @@ def phase_table(ci, launch, L, batch):
     return out
 
 
+def run_prefill_only(args, cfg):
+    """The pre-fill stage alone on a few layers: activations (tensor cores; synthesised for the planted
+    configuration), selection, compaction.  The target of ncu captures of those kernels."""
+    import torch
+    import paper_2410_18311_b200 as ci
+    from paper_2410_18311_b200 import _build, workloads as wl
+    _build.build()
+    L = args.prefill_only
+    kind = ci.FFN_RELU_GATED if cfg.gated else ci.FFN_RELU
+    K = ci.coreinfer_count(cfg.beta, cfg.d_ff)
+    X = wl.prompt_hidden(cfg, device="cuda")
+    weights = [wl.layer_weights(cfg, l, device="cuda") for l in range(L)]
+    A = torch.empty((cfg.T, cfg.d_ff), device="cuda")
+    S = torch.empty(K, dtype=torch.int32, device="cuda")
+    tws = torch.empty(ci.coreinfer_prefill_activations_workspace_bytes(), dtype=torch.uint8, device="cuda")
+    sws = torch.empty(ci.coreinfer_select_workspace_bytes(cfg.T, cfg.d_ff), dtype=torch.uint8, device="cuda")
+    new = lambda: torch.empty((K, cfg.d_model), dtype=cfg.torch_dtype, device="cuda")
+    up_c, down_c, gate_c = new(), new(), (new() if cfg.gated else None)
+    planted = [wl.planted_activations(cfg, l, cfg.T, device="cuda")[0] for l in range(L)] if cfg.planted else None
+    stream = torch.cuda.current_stream()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    t = [0.0, 0.0, 0.0]
+
+    def step(timed):
+        for l in range(L):
+            w_up, w_gate, w_down = weights[l]
+            ev[0].record(stream)
+            if cfg.planted:
+                act = planted[l]
+            else:
+                ci.coreinfer_prefill_activations(X, kind, w_up, w_gate, None, A, tws, stream)
+                act = A
+            ev[1].record(stream)
+            ci.coreinfer_select_core(act, cfg.alpha, cfg.beta, S, None, sws, stream)
+            ev[2].record(stream)
+            ci.coreinfer_compact(w_up, w_gate, w_down, None, S, K, up_c, gate_c, down_c, None, stream)
+            ev[3].record(stream)
+            if timed:
+                torch.cuda.synchronize()
+                for i in range(3):
+                    t[i] += ev[i].elapsed_time(ev[i + 1])
+    for _ in range(args.warmup):
+        step(False)
+    torch.cuda.synchronize()
+    for _ in range(args.steps):
+        step(True)
+    ci.coreinfer_workspace_status(sws)
+    n = args.steps * L
+    print(json.dumps({"mode": "prefill-only", "workload": cfg.name, "layers": L, "T": cfg.T, "K": K,
+                      "activations_us_per_layer": None if cfg.planted else 1e3 * t[0] / n,
+                      "select_us_per_layer": 1e3 * t[1] / n, "compact_us_per_layer": 1e3 * t[2] / n}), flush=True)
+
+
 def main():
     args = parse_args()
     from paper_2410_18311_b200 import workloads as wl
     cfg = wl.CONFIGS[args.config]
+    if args.prefill_only > 0:
+        return run_prefill_only(args, cfg)
     if args.decode_only > 0:
         return run_decode_only(args, cfg)
     if args.impl == "reference":
