@@ -16,10 +16,12 @@
 // per-row costs of a warp are one sixteen-byte load per vector and its multiply-adds.
 //
 // Exchange per layer: the CTA's partial y (d_model fp32) is assembled in shared memory and added
-// into a global vector with one bulk reduction; one thread waits for it, arrives at a grid
-// barrier (release), polls for everybody else's arrival (acquire) and brings the sum back with
-// one bulk copy, on whose barrier the other consumers sleep; every thread then forms its columns
-// of the next layer's input.  While the exchange is on, the producer requests only a limited
+// into a global vector with one bulk reduction; one lane of a third kind of warp, the exchange
+// warp, waits for it, arrives at a grid barrier (release), polls for everybody else's arrival
+// (acquire) and brings the sum back with one bulk copy, on whose barrier the consumers sleep --
+// after they have pulled the first two batches of the next layer into their register buffers,
+// which frees two more batch slots for the producer; every thread then forms its columns of the
+// next layer's input.  While the exchange is on, the producer requests only a limited
 // number of rows: a first part before the exchange (landed by then), a second part once this
 // CTA's arrival is out (a fence waits for the SM's bulk copies in flight, so none is issued
 // before), paced.  Every wait (slot barriers, grid barrier, read-back) is bounded: when one gives
@@ -283,7 +285,7 @@ __device__ __forceinline__ float warp_reduce_n(const float (&v)[4], int lane) { 
 // k0 .. k1-1.  Each of the two phases is cut into batches of BATCH rows (the last one of a phase
 // may hold fewer); every batch takes one batch slot of the ring, whatever it holds.
 template <typename T, int VPT, bool GATED>
-__global__ void __launch_bounds__(max_consumers(VPT) + 32, 1)
+__global__ void __launch_bounds__(max_consumers(VPT) + 64, 1)
 decode_stack_kernel(const __grid_constant__ DecodeParams p)
 {
     using E = Elem<T>;
@@ -331,7 +333,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
     // Eight lanes issue copies: one round fills up to 8 / BATCH consecutive batch slots, lane j
     // taking row j % BATCH of batch j / BATCH of the round.  Every lane waits for its batch slot to
     // be free; the lane of the batch's first row announces the bytes of the whole batch.
-    if (tid >= NC) {
+    if (tid >= NC && tid < NC + 32) {
         const int lane = tid - NC;
         constexpr int RB = 8 / BATCH;
         const int round_max = NB < RB ? NB : RB;
@@ -433,6 +435,47 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
         return;
     }
 
+    // ======================================================== exchange warp ==
+    // One lane runs every layer's exchange, so that all consumer warps are free to pull the
+    // first batches of the next layer into their registers meanwhile: it waits (CTA barrier 2)
+    // until the consumers have assembled the CTA's partial y in shared memory, sends it as one
+    // bulk reduction and waits for that, arrives at the grid barrier (a release: the consumers'
+    // earlier plain writes to global memory, such as the cleared target of a later layer, are
+    // known to this thread through the CTA barrier), waits for everybody else's arrival, and
+    // issues the copy that brings the sum back into the same buffer; the consumers sleep on that
+    // copy's barrier.
+    if (tid >= NC + 32) {
+        const int lane = tid - NC - 32;
+        unsigned long long* const stamps = lane == 0 ? p.stamps : nullptr;
+        for (int l = 0; l < p.L; ++l) {
+            named_bar_sync(2, NC + 32);
+            if (lane == 0) {
+                const size_t sb = ((size_t)cta * p.L + l) * kStampSlots;
+                (void)sb;
+                float* ytarget = p.ybuf + (size_t)(l % kYBuffers) * p.d;
+                CI_STAMP(stamps, sb, 4);
+                if (!*abort_flag) {
+                    bulk_reduce_add_f32(ytarget, smem_u32(ysum), (uint32_t)p.d * (uint32_t)sizeof(float));
+                    bulk_wait_all();
+                    CI_STAMP(stamps, sb, 5);
+                    red_release_add(&p.ctrl[1], 1u);
+                    *arrived = l + 1;         // the fence is behind us: the producer may go on, paced
+                    CI_STAMP(stamps, sb, 6);
+                    grid_wait(p.ctrl, (unsigned)(l + 1) * (unsigned)G, abort_flag);
+                    CI_STAMP(stamps, sb, 7);
+                }
+                if (!*abort_flag) {
+                    const uint32_t yb = smem_u32(y_bar);
+                    mbar_arrive_expect_tx(yb, (uint32_t)p.d * (uint32_t)sizeof(float));
+                    bulk_g2s(smem_u32(ysum), ytarget, (uint32_t)p.d * (uint32_t)sizeof(float), yb);
+                    *layers_done = l + 1;     // the exchange's last request is on its way: the producer may go on freely
+                }
+            }
+            __syncwarp();
+        }
+        return;
+    }
+
     // ============================================================ consumers ==
     const int lane = tid & 31;
     const int warp = tid >> 5;
@@ -474,7 +517,22 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
         if (++bslot == NB) { bslot = 0; phase ^= 1u; }
     };
 
-    unsigned long long* const stamps = tid == 0 ? p.stamps : nullptr;   // thread 0 runs the exchange
+    unsigned long long* const stamps = tid == 0 ? p.stamps : nullptr;
+    // The two register buffers live across layers: while the exchange of layer l is on, the
+    // first two batches of layer l + 1 are pulled into them (their slots are free for the
+    // producer at once), so a layer starts with up to two batches in registers besides the ring.
+    uint4 qa[BATCH][VPT], qb[BATCH][VPT];
+    auto batches_of = [&](int l) {
+        int k0, k1;
+        slab_of(cta, G, l, p.layers[l].K, &k0, &k1);
+        const int n = k1 - k0;
+        return (n * NMAT + BATCH - 1) / BATCH + (n + BATCH - 1) / BATCH;
+    };
+    {
+        const int nb0 = batches_of(0);
+        if (nb0 > 0) fetch(qa);
+        if (nb0 > 1) fetch(qb);
+    }
     for (int l = 0; l < p.L; ++l) {
         const LayerDev& ly = p.layers[l];
         int k0, k1;
@@ -567,13 +625,12 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
         };
 
         {
-            uint4 qa[BATCH][VPT], qb[BATCH][VPT];
-            if (nbt > 0) fetch(qa);
+            // on entry qa holds batch 0 and qb batch 1 of this layer (where they exist)
             for (int b = 0; b < nbt; b += 2) {
-                if (b + 1 < nbt) fetch(qb);
                 process(qa, b, 0);
                 if (b + 2 < nbt) fetch(qa);
                 if (b + 1 < nbt) process(qb, b + 1, 1);
+                if (b + 3 < nbt) fetch(qb);
             }
             if (nbt == 0) {                          // a CTA without neurons still meets the others at the barriers
                 named_bar_sync(1, NC);
@@ -587,7 +644,6 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
         // reads the sum back.  Targets rotate over three buffers: while layer l's is read, the
         // one layer l+2 will use is cleared (last read before the barrier of l).
         const bool last = (l == p.L - 1);
-        float* ytarget = p.ybuf + (size_t)(l % kYBuffers) * d;
         // One sum per CTA leaves the chip, as one bulk reduction from shared memory (L2 then
         // sees 128-byte line reductions instead of a thousand 16-byte atomics per CTA).
 #pragma unroll
@@ -601,31 +657,12 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
             }
         }
         fence_proxy_async();          // these generic-proxy writes are read by the copy engine next
-        named_bar_sync(1, NC);
-        // One thread runs the exchange: the CTA's reduction and the wait for its completion, the
-        // arrival at the grid barrier (a release: the CTA's earlier plain writes to global memory,
-        // such as the cleared target of a later layer, are known to this thread through the CTA
-        // barriers since), the wait for everybody else's arrival, and the copy that brings the
-        // sum back into the buffer the partial left from; the other consumers sleep on that
-        // copy's barrier.
-        if (tid == 0) {
-            CI_STAMP(stamps, sb, 4);
-            if (!*abort_flag) {
-                bulk_reduce_add_f32(ytarget, smem_u32(ysum), (uint32_t)d * (uint32_t)sizeof(float));
-                bulk_wait_all();
-                CI_STAMP(stamps, sb, 5);
-                red_release_add(&p.ctrl[1], 1u);
-                *arrived = l + 1;         // the fence is behind us: the producer may trickle
-                CI_STAMP(stamps, sb, 6);
-                grid_wait(p.ctrl, (unsigned)(l + 1) * (unsigned)G, abort_flag);
-                CI_STAMP(stamps, sb, 7);
-            }
-            if (!*abort_flag) {
-                const uint32_t yb = smem_u32(y_bar);
-                mbar_arrive_expect_tx(yb, (uint32_t)d * (uint32_t)sizeof(float));
-                bulk_g2s(smem_u32(ysum), ytarget, (uint32_t)d * (uint32_t)sizeof(float), yb);
-                *layers_done = l + 1;     // the exchange's last request is on its way: the producer may go on
-            }
+        named_bar_arrive(2, NC + 32);  // hands the partial to the exchange warp; nobody waits here
+        // while the exchange runs: the first two batches of the next layer into the registers
+        if (!last) {
+            const int nbn = batches_of(l + 1);
+            if (nbn > 0) fetch(qa);
+            if (nbn > 1) fetch(qb);
         }
         wait_slot(smem_u32(y_bar), (uint32_t)(l & 1), abort_flag, p.ctrl);
         CI_STAMP(stamps, sb, 8);
@@ -712,7 +749,7 @@ static coreinfer_status launch_one(const DecodeParams& p, int grid, size_t smem,
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3((unsigned)(p.nc + 32));
+    cfg.blockDim = dim3((unsigned)(p.nc + 64));    // consumers, producer warp, exchange warp
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -838,15 +875,21 @@ static coreinfer_status decode_stack_b1(const coreinfer_layer* layers, int L, co
     p.n_bslots = (int)bslots;
     const size_t smem = fixed + (size_t)p.n_bslots * bslot_bytes;
     // While an exchange is on, the next layer's rows are requested in two parts (measured on the
-    // four model shapes): about 72 KB ahead of the exchange -- more would still be in flight when
-    // the CTA's fence runs, and a fence waits for the SM's own copies in flight -- and the rest of
-    // the ring after the CTA's arrival, one batch per 1400 cycles and 32 KB, which is about the pace
-    // at which HBM serves one SM.
-    const int rows_ahead = 72 * 1024 / p.slot_bytes;
+    // four model shapes): about 100 KB ahead of the exchange (40 KB for rows wider than 12 KB) --
+    // more would still be in flight when the CTA's fence runs, and a fence waits for the SM's own
+    // copies in flight -- and the rest of the ring after the CTA's arrival, one batch per 1000
+    // cycles and 32 KB, which is a little above the pace at which HBM serves one SM.
+    const int rows_ahead = (p.slot_bytes <= 12 * 1024 ? 100 : 40) * 1024 / p.slot_bytes;
     p.runahead = rows_ahead / batch < 1 ? 1 : rows_ahead / batch;
     if (p.runahead > p.n_bslots) p.runahead = p.n_bslots;
-    p.trickle = p.n_bslots - p.runahead;
-    p.trickle_gap = (int)(1400ll * (long long)bslot_bytes / 32768);
+    p.trickle = p.n_bslots - p.runahead + 2;     // + the two slots the consumers empty into their registers meanwhile
+    p.trickle_gap = (int)(1000ll * (long long)bslot_bytes / 32768);
+#ifdef COREINFER_TUNE
+    { const char* e;
+      if ((e = getenv("X_RUNAHEAD"))) p.runahead = atoi(e);
+      if ((e = getenv("X_TRICKLE"))) p.trickle = atoi(e);
+      if ((e = getenv("X_GAP"))) p.trickle_gap = atoi(e); }
+#endif
     p.ysum_ofs = (int)((size_t)p.n_bslots * bslot_bytes + fixed0);
     p.x0 = x0;
     p.y_last = y_last;
