@@ -327,6 +327,7 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
         *arrived = 0;
         mbar_fence_init();
     }
+    if (tid < kMaxWarps) ss_red[tid] = 0.f;
     __syncthreads();
 
     // ======================================================== producer warp ==
@@ -707,7 +708,14 @@ decode_stack_kernel(const __grid_constant__ DecodeParams p)
         if (lane == 0) ss_red[warp] = ss;
         named_bar_sync(1, NC);
         float tot = 0.f;
-        for (int w = 0; w < nwarps; ++w) tot += ss_red[w];
+        {   // the warps' sums (entries beyond the last warp are zero): four 16-byte loads, same order in every thread
+            const float4* s4 = reinterpret_cast<const float4*>(ss_red);
+#pragma unroll
+            for (int w = 0; w < kMaxWarps / 4; ++w) {
+                const float4 t = s4[w];
+                tot += (t.x + t.y) + (t.z + t.w);
+            }
+        }
         const float inv = rsqrtf(tot * p.inv_d);     // within 2 ulp of 1 / sqrt(mean square)
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
@@ -848,7 +856,7 @@ static coreinfer_status decode_stack_b1(const coreinfer_layer* layers, int L, co
         p.layers[l].pad = 0;
         if (layers[l].K > Kmax) Kmax = layers[l].K;
     }
-    p.rmax = (Kmax + G - 1) / G + 1;
+    p.rmax = ((Kmax + G - 1) / G + 1 + 3) & ~3;     // a multiple of 4 keeps the arrays behind it 16-byte aligned
     if ((unsigned long long)Kmax * (unsigned long long)G >= (1ull << 32))
         CI_FAIL(COREINFER_ERR_UNSUPPORTED, "K = %d is too large for the slab split (K * SM count must stay below 2^32)", Kmax);
     p.inv_d = 1.0f / (float)d_model;
