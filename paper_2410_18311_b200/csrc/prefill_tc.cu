@@ -3,9 +3,9 @@
 // obtains it as a by-product of the dense pre-fill pass, Section 4.2 / Fig. 1).  bf16 or fp16 inputs,
 // exact products, fp32 accumulation in tensor memory, fp32 output.
 //
-// One persistent CTA per SM walks 128 x 128 output tiles.  Warp 0 (one lane) feeds a ring of
+// One persistent CTA per SM walks output tiles of 128 prompt rows x 256 neurons (128 when gated).  Warp 0 (one lane) feeds a ring of
 // shared-memory stages with 2-D tensor copies (128-byte swizzle, each stage a 128 x 64 slice of X
-// and of the weight matrices); warp 1 (one lane) issues tcgen05.mma (M 128, N 128, K 16, four per
+// and a 256 (128) x 64 slice of each weight matrix); warp 1 (one lane) issues tcgen05.mma (M 128, N 256 or 128, K 16, four per
 // stage and matrix) into one of two accumulator sets in tensor memory and hands stages back
 // through tcgen05.commit; warps 2..5 read a finished accumulator set (tcgen05.ld, 32 columns at a
 // time, each thread one output row), apply bias / ReLU / gate product and store, while the MMA
@@ -19,7 +19,9 @@
 namespace coreinfer {
 
 constexpr int kTcBM = 128;                 // prompt rows per tile
-constexpr int kTcBN = 128;                 // neurons per tile
+// neurons per tile: 256 (the widest MMA) where one weight matrix is multiplied, 128 where the gate
+// matrix doubles the accumulators (two sets of 2 x 128 columns fill the 512 columns of tensor memory)
+__host__ __device__ constexpr int tc_bn(bool gated) { return gated ? 128 : 256; }
 constexpr int kTcBK = 64;                  // reduction slice per stage: 128 bytes of bf16 = one swizzle row
 constexpr int kTcUmmaK = 16;
 constexpr int kTcThreads = 192;            // warp 0 copies, warp 1 MMA + tensor memory, warps 2..5 epilogue
@@ -126,9 +128,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                   const __grid_constant__ CUtensorMap map_gate, const TcParams p)
 {
     constexpr int NB = GATED ? 2 : 1;                          // weight matrices per stage
-    constexpr uint32_t STAGE_BYTES = (1 + NB) * kTcTileBytes;
+    constexpr int kTcBN = tc_bn(GATED);
+    constexpr uint32_t W_TILE_BYTES = (uint32_t)kTcBN * kTcBK * 2;     // one weight slice: kTcBN rows of 128 bytes
+    constexpr uint32_t STAGE_BYTES = kTcTileBytes + NB * W_TILE_BYTES;
     constexpr uint32_t ACC_COLS = NB * kTcBN;                  // tensor-memory columns of one accumulator set
-    constexpr uint32_t TMEM_COLS = 2 * ACC_COLS;               // two sets: 256 or 512 columns
+    constexpr uint32_t TMEM_COLS = 2 * ACC_COLS;               // two sets: 512 columns
     const uint32_t IDESC = p.idesc;
 
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -181,7 +185,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                     mbar_arrive_expect_tx(fb, STAGE_BYTES);
                     tensor_g2s_2d(dst, &map_x, kb * kTcBK, m0, fb);
                     tensor_g2s_2d(dst + kTcTileBytes, &map_up, kb * kTcBK, n0, fb);
-                    if (GATED) tensor_g2s_2d(dst + 2 * kTcTileBytes, &map_gate, kb * kTcBK, n0, fb);
+                    if (GATED) tensor_g2s_2d(dst + kTcTileBytes + W_TILE_BYTES, &map_gate, kb * kTcBK, n0, fb);
                     if (++s == p.stages) { s = 0; ph ^= 1u; }
                 }
             }
@@ -205,7 +209,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                     const uint32_t base = smem_u32(tiles + (size_t)s * STAGE_BYTES);
                     const uint64_t da = smem_desc_k_sw128(base);
                     const uint64_t db = smem_desc_k_sw128(base + kTcTileBytes);
-                    const uint64_t dg = smem_desc_k_sw128(base + 2 * kTcTileBytes);
+                    const uint64_t dg = smem_desc_k_sw128(base + kTcTileBytes + W_TILE_BYTES);
 #pragma unroll
                     for (int k4 = 0; k4 < kTcBK / kTcUmmaK; ++k4) {
                         const uint32_t acc = (kb > 0 || k4 > 0) ? 1u : 0u;
@@ -308,15 +312,15 @@ static coreinfer_status encode_fn(EncodeTiledFn* out)
     return COREINFER_OK;
 }
 
-// [rows][cols] bf16 or fp16 row-major, read in boxes of 128 rows x 64 columns with the 128-byte swizzle.
-static coreinfer_status make_map(CUtensorMap* map, const void* base, int rows, int cols, bool f16)
+// [rows][cols] bf16 or fp16 row-major, read in boxes of `box_rows` rows x 64 columns with the 128-byte swizzle.
+static coreinfer_status make_map(CUtensorMap* map, const void* base, int rows, int cols, bool f16, int box_rows)
 {
     EncodeTiledFn enc;
     coreinfer_status s = encode_fn(&enc);
     if (s != COREINFER_OK) return s;
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)kTcBK, (cuuint32_t)kTcBM};
+    const cuuint32_t box[2] = {(cuuint32_t)kTcBK, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     const CUresult r = enc(map, f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -362,9 +366,10 @@ coreinfer_status coreinfer_prefill_activations(const void* x, int32_t T, coreinf
     cudaStream_t st = (cudaStream_t)cuda_stream;
 
     CUtensorMap map_x, map_up, map_gate;
-    if ((s = make_map(&map_x, x, T, d_model, f16)) != COREINFER_OK) return s;
-    if ((s = make_map(&map_up, w_up, d_ff, d_model, f16)) != COREINFER_OK) return s;
-    if ((s = make_map(&map_gate, gated ? w_gate : w_up, d_ff, d_model, f16)) != COREINFER_OK) return s;
+    const int kTcBN = tc_bn(gated);
+    if ((s = make_map(&map_x, x, T, d_model, f16, kTcBM)) != COREINFER_OK) return s;
+    if ((s = make_map(&map_up, w_up, d_ff, d_model, f16, kTcBN)) != COREINFER_OK) return s;
+    if ((s = make_map(&map_gate, gated ? w_gate : w_up, d_ff, d_model, f16, kTcBN)) != COREINFER_OK) return s;
 
     TcParams p;
     p.T = T;
@@ -383,7 +388,7 @@ coreinfer_status coreinfer_prefill_activations(const void* x, int32_t T, coreinf
     p.out = act_out;
     p.bias = b_up;
     p.status = (unsigned*)workspace;
-    const size_t stage = (size_t)(gated ? 3 : 2) * kTcTileBytes;
+    const size_t stage = (size_t)kTcTileBytes + (size_t)(gated ? 2 : 1) * kTcBN * kTcBK * 2;
     const size_t fixed = 1024 /* alignment slack */ + (2 * kTcMaxStages + 4) * sizeof(uint64_t) + 64;
     long long stages = ((long long)di.smem_optin - (long long)fixed) / (long long)stage;
     if (stages > kTcMaxStages) stages = kTcMaxStages;
