@@ -149,7 +149,8 @@ coreinfer_status coreinfer_verify_core_idx(const int32_t* core_idx, int32_t K, i
  *   b_up_c     device [K] in `dtype` or NULL (RELU only); b_down device [d_model] in `dtype` or NULL
  *   y          device out [batch, d_model] fp32
  *   workspace  device scratch of at least coreinfer_ffn_decode_workspace_bytes().
- * 1 <= batch <= COREINFER_MAX_BATCH.
+ * 1 <= batch <= COREINFER_MAX_BATCH.  At batch 1 a row (d_model elements) may take up to 21504 bytes
+ * (d_model <= 10752 in bf16 / fp16, 5376 in fp32); wider rows return UNSUPPORTED.
  * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA. */
 size_t coreinfer_ffn_decode_workspace_bytes(int32_t batch, int32_t d_model, int32_t K);
 
@@ -222,8 +223,8 @@ coreinfer_status coreinfer_ffn_decode_stack(const coreinfer_layer* layers, int32
  * Arguments and results are those of coreinfer_ffn_decode_stack without the workspace pair,
  * for batch 1 only (any other batch returns COREINFER_ERR_UNSUPPORTED).
  * Limit: the scratch the kernel needs, 256 + 12 * d_model bytes (any number of layers), must fit
- * in 128 KiB, i.e. d_model <= 10901; wider models return COREINFER_ERR_UNSUPPORTED and enqueue
- * nothing -- use the workspace variant for them.
+ * in 128 KiB, i.e. d_model <= 10901 (which covers every row width the batch-1 kernel takes); wider
+ * models return COREINFER_ERR_UNSUPPORTED and enqueue nothing.
  * The first call on each device looks up the array's device address (cudaGetSymbolAddress),
  * which is set-up work rather than stream work: make that first call before starting any
  * stream capture.

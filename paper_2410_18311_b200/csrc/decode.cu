@@ -892,12 +892,6 @@ static coreinfer_status decode_stack_b1(const coreinfer_layer* layers, int L, co
     if (p.runahead > p.n_bslots) p.runahead = p.n_bslots;
     p.trickle = p.n_bslots - p.runahead + 2;     // + the two slots the consumers empty into their registers meanwhile
     p.trickle_gap = (int)(1000ll * (long long)bslot_bytes / 32768);
-#ifdef COREINFER_TUNE
-    { const char* e;
-      if ((e = getenv("X_RUNAHEAD"))) p.runahead = atoi(e);
-      if ((e = getenv("X_TRICKLE"))) p.trickle = atoi(e);
-      if ((e = getenv("X_GAP"))) p.trickle_gap = atoi(e); }
-#endif
     p.ysum_ofs = (int)((size_t)p.n_bslots * bslot_bytes + fixed0);
     p.x0 = x0;
     p.y_last = y_last;
