@@ -506,6 +506,7 @@ def run_ours(args, cfg):
         pre["select_floor_us_at_measured_peak"] = pre["activation_bytes"] / peak / 1e3
         line["prefill_stage_one_layer"] = pre
         line["configs"] = other_configs(ci, wl, peak, cfg.name)
+        line["extensions"] = extension_times(ci, wl, peak)
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = oracle_sample(cfg, n_layers=4, n_tokens=min(cfg.decode_steps, 256))
     print(json.dumps(line), flush=True)
@@ -584,6 +585,65 @@ def prefill_stage_times(ci, wl, cfg, T, beta, layer=0):
                                    2.0 * T * cfg.d_model * cfg.d_ff * (2 if cfg.gated else 1) / act_us / 1e6),
             "select_us": 1e3 * sel, "select_floor_us_at_measured_peak": None,
             "activation_bytes": 4 * T * cfg.d_ff, "compact_us": 1e3 * cmp_}
+
+
+def extension_times(ci, wl, peak):
+    """The calls beyond the timed path, at the headline shapes: the SiLU-gated / fp16 decode stack
+    (Llama-2-7B shape), and the set calls (top fraction by count, similarity, nearest centroid,
+    in-place update of 5 % of a deployed OPT-6.7B-shaped layer)."""
+    import numpy as np
+    import torch
+    out = {}
+    cfg = wl.CONFIGS["relu-llama2-7b"]
+    K = ci.coreinfer_count(cfg.beta, cfg.d_ff)
+    w = [tuple(t if t is None else t.to(torch.float16) for t in wl.compacted_weights_random(cfg, l, K, device="cuda"))
+         for l in range(cfg.L)]
+    arr = ci.binding.make_layers([(u, g, dn, None, None) for (u, g, dn) in w])
+    xs = [wl.decode_input(cfg, s, device="cuda").to(torch.float16) for s in range(16)]
+    y = torch.empty((1, cfg.d_model), device="cuda")
+    ws = torch.empty(ci.coreinfer_ffn_decode_stack_workspace_bytes(cfg.L, 1, cfg.d_model, K), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+    ms = _time_ms(lambda: [ci.coreinfer_ffn_decode_stack(arr, xs[t], ci.FFN_SILU_GATED, y, None, None, ws, stream)
+                           for t in range(16)], stream, 3) / 16
+    ci.coreinfer_workspace_status(ws)
+    nbytes = cfg.L * 3 * K * cfg.d_model * 2
+    out["silu_gated_fp16_decode_llama_shape"] = {"us_per_layer": 1e3 * ms / cfg.L, "tok_s": 1e3 / ms,
+                                                 "gbs": nbytes / ms / 1e6, "frac_of_measured": nbytes / ms / 1e6 / peak}
+    del w, arr
+    torch.cuda.empty_cache()
+    c2 = wl.CONFIGS["opt6.7b"]
+    N, K2 = c2.d_ff, ci.coreinfer_count(c2.beta, c2.d_ff)
+    g = torch.Generator(device="cuda").manual_seed(1)
+    counts = torch.randint(0, c2.T + 1, (N,), generator=g, device="cuda", dtype=torch.int32)
+    S = torch.empty(K2, dtype=torch.int32, device="cuda")
+    out["top_by_count_us"] = 1e3 * _time_ms(lambda: ci.coreinfer_top_by_count(counts, c2.T, c2.beta, S, stream), stream, 20)
+    rng = np.random.default_rng(0)
+    S0 = np.sort(rng.choice(N, size=K2, replace=False)).astype(np.int32)
+    keep = rng.choice(S0, size=K2 - K2 // 20, replace=False)
+    S1 = np.sort(np.concatenate([keep, rng.choice(np.setdiff1d(np.arange(N), S0), size=K2 - len(keep), replace=False)])).astype(np.int32)
+    a, b = torch.from_numpy(S0).cuda(), torch.from_numpy(S1).cuda()
+    pair = torch.empty(2, dtype=torch.int32, device="cuda")
+    out["core_similarity_us"] = 1e3 * _time_ms(lambda: ci.coreinfer_core_similarity(a, b, pair, stream), stream, 20)
+    C = torch.randn((16, c2.d_model), generator=g, device="cuda")
+    v = torch.randn((c2.d_model,), generator=g, device="cuda")
+    cws = torch.empty(ci.coreinfer_nearest_centroid_workspace_bytes(16), dtype=torch.uint8, device="cuda")
+    gi = torch.empty(1, dtype=torch.int32, device="cuda")
+    out["nearest_centroid_16_groups_us"] = 1e3 * _time_ms(lambda: ci.coreinfer_nearest_centroid(C, v, gi, cws, stream), stream, 20)
+    w_up, _, w_down = wl.layer_weights(c2, 0, device="cuda")
+    new = lambda: torch.empty((K2, c2.d_model), dtype=c2.torch_dtype, device="cuda")
+    up_c, down_c = new(), new()
+    ci.coreinfer_compact(w_up, None, w_down, None, a, K2, up_c, None, down_c, None, stream)
+    uws = torch.empty(ci.coreinfer_update_core_set_workspace_bytes(N, K2), dtype=torch.uint8, device="cuda")
+    nch = torch.empty(1, dtype=torch.int32, device="cuda")
+    slot = a.clone()
+    sets = [b, a]
+
+    def flip(i=[0]):          # alternate between the two sets: every call rewrites 5 % of the rows
+        ci.coreinfer_update_core_set(w_up, None, w_down, None, slot, sets[i[0] & 1], up_c, None, down_c, None, nch, uws, stream)
+        i[0] += 1
+    out["update_core_set_5pct_us"] = 1e3 * _time_ms(flip, stream, 10)
+    out["update_core_set_rows_changed"] = int(nch.item())
+    return out
 
 
 def other_configs(ci, wl, peak, headline):

@@ -158,3 +158,40 @@ def test_two_group_stack_with_odd_slabs():
         layers = _rand_layers(d, Ks, gated, torch.bfloat16, 9000 + d, bias=not gated)
         x0 = torch.randn(1, d, generator=torch.Generator().manual_seed(d + 1)).to(torch.bfloat16).cuda()
         check_stack_teacher_forced(layers, x0, ci.FFN_RELU_GATED if gated else ci.FFN_RELU, torch.bfloat16)
+
+
+@pytest.mark.parametrize("dtype,kind", [(torch.float16, "silu"), (torch.bfloat16, "silu"), (torch.float16, "relu_gated")])
+def test_llama_shaped_layer_with_silu_gate_and_fp16(dtype, kind):
+    """One full-size Llama-2-7B-shaped layer (d_model 4096, d_ff 11008, T 1024) of the second
+    workload family: tensor-core activations with the SiLU gate, selection on them (they carry
+    negative entries), compaction, decode at 1 and 8 sequences; and eight layers of the stack."""
+    require_gpu()
+    cfg = wl.CONFIGS["relu-llama2-7b"]
+    k = ci.FFN_SILU_GATED if kind == "silu" else ci.FFN_RELU_GATED
+    X = wl.prompt_hidden(cfg, device="cuda").to(dtype)
+    w_up, w_gate, w_down = (t.to(dtype) for t in wl.layer_weights(cfg, 5, device="cuda"))
+    A = torch.empty((cfg.T, cfg.d_ff), device="cuda")
+    tws = torch.empty(ci.coreinfer_prefill_activations_workspace_bytes(), dtype=torch.uint8, device="cuda")
+    ci.coreinfer_prefill_activations(X, k, w_up, w_gate, None, A, tws)
+    ci.coreinfer_workspace_status(tws)
+    rows = [0, 500, cfg.T - 1]
+    H_o, _ = oracle.ffn_dense(to_f32_np(X[rows]), k, to_f32_np(w_up), to_f32_np(w_gate),
+                              np.zeros((cfg.d_model, cfg.d_ff), np.float32), want_y=False)
+    assert_ffn_close(A[rows].cpu().numpy(), H_o, torch.float32)
+    S, f = gpu_select(A, cfg.alpha, cfg.beta)
+    S_o, f_o = oracle.select(A.cpu().numpy(), cfg.alpha, cfg.beta)
+    np.testing.assert_array_equal(f, f_o)
+    np.testing.assert_array_equal(S, S_o)
+    up_c, gate_c, down_c, _ = gpu_compact(w_up, w_gate, w_down, None, torch.from_numpy(S).cuda())
+    o_up, o_gate, o_down, _ = oracle.compact(raw_np(w_up), raw_np(w_gate), raw_np(w_down), None, S_o)
+    assert raw_np(up_c).tobytes() == o_up.tobytes() and raw_np(gate_c).tobytes() == o_gate.tobytes()
+    assert raw_np(down_c).tobytes() == o_down.tobytes()
+    for B in (1, 8):
+        x = wl.decode_input(cfg, 3, device="cuda", batch=B).to(dtype)
+        y = gpu_decode(x, k, up_c, gate_c, down_c)
+        y_o = oracle.ffn(to_f32_np(x), k, to_f32_np(up_c), to_f32_np(gate_c), to_f32_np(down_c))
+        assert_ffn_close(y, y_o, dtype)
+    K = len(S)
+    layers = [tuple(t if t is None else t.to(dtype) for t in wl.compacted_weights_random(cfg.with_(L=8), l, K, device="cuda")) + (None, None)
+              for l in range(8)]
+    check_stack_teacher_forced(layers, wl.decode_input(cfg, 0, device="cuda").to(dtype), k, dtype, layers_to_check=(0, 3, 7))

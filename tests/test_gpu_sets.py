@@ -153,3 +153,31 @@ def test_update_core_set_in_place(dtype, gated):
         y = gpu_decode(x, kind, up_c, gate_c, down_c, bup_c)
         y_o = oracle.ffn(to_f32_np(x), kind, to_f32_np(up_c), to_f32_np(gate_c), to_f32_np(down_c), to_f32_np(bup_c))
         assert_ffn_close(y, y_o, dtype)
+
+
+def test_update_core_set_at_the_opt67b_shape():
+    """A deployed OPT-6.7B-shaped layer (d_model 4096, d_ff 16384, K 3277) whose set changes by 5 %:
+    pairs as the oracle lists them, buffers equal to a fresh compaction of the new set row for row."""
+    require_gpu()
+    cfg = wl.CONFIGS["opt6.7b"]
+    w_up, _, w_down = wl.layer_weights(cfg, 1, device="cuda")
+    N, K = cfg.d_ff, ci.coreinfer_count(cfg.beta, cfg.d_ff)
+    rng = np.random.default_rng(8)
+    S0 = np.sort(rng.choice(N, size=K, replace=False)).astype(np.int32)
+    up_c, _, down_c, _ = gpu_compact(w_up, None, w_down, None, torch.from_numpy(S0).cuda())
+    keep = rng.choice(S0, size=K - K // 20, replace=False)
+    S1 = np.sort(np.concatenate([keep, rng.choice(np.setdiff1d(np.arange(N), S0), size=K - len(keep), replace=False)])).astype(np.int32)
+    slot_neuron = torch.from_numpy(S0.copy()).cuda()
+    ws = torch.empty(ci.coreinfer_update_core_set_workspace_bytes(N, K), dtype=torch.uint8, device="cuda")
+    nch = torch.zeros(1, dtype=torch.int32, device="cuda")
+    sim = torch.zeros(2, dtype=torch.int32, device="cuda")
+    ci.coreinfer_core_similarity(torch.from_numpy(S0).cuda(), torch.from_numpy(S1).cuda(), sim)
+    ci.coreinfer_update_core_set(w_up, None, w_down, None, slot_neuron, torch.from_numpy(S1).cuda(), up_c, None, down_c, None, nch, ws)
+    torch.cuda.synchronize()
+    assert tuple(sim.cpu().tolist()) == oracle.core_similarity(S0, S1) == (len(keep), 2 * K - len(keep))
+    slots_o, neurons_o, slot_o = oracle.set_delta(S0, S1)
+    assert int(nch.item()) == len(slots_o) == K // 20
+    np.testing.assert_array_equal(slot_neuron.cpu().numpy(), slot_o)
+    o_up, _, o_down, _ = oracle.compact(raw_np(w_up), None, raw_np(w_down), None, S1)
+    perm = np.argsort(slot_o, kind="stable")
+    assert raw_np(up_c)[perm].tobytes() == o_up.tobytes() and raw_np(down_c)[perm].tobytes() == o_down.tobytes()
