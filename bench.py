@@ -29,7 +29,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode_stack_kernel launch at the bench
 # workload, from an ncu capture of a 4-layer launch of the same shapes scaled by the layer count
 # (every layer streams its own weights).  None whenever the kernel has changed since the capture.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"opt6.7b": 219.59e6 / 4 * 32}
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"opt6.7b": 219.17e6 / 4 * 32}
 
 
 def parse_args():
