@@ -19,9 +19,14 @@
 namespace coreinfer {
 
 constexpr int kTcBM = 128;                 // prompt rows per tile
-// neurons per tile: 256 (the widest MMA) where one weight matrix is multiplied, 128 where the gate
-// matrix doubles the accumulators (two sets of 2 x 128 columns fill the 512 columns of tensor memory)
-__host__ __device__ constexpr int tc_bn(bool gated) { return gated ? 128 : 256; }
+// Neurons per tile: up to 256 (the widest MMA) where one weight matrix is multiplied, up to 128
+// where the gate matrix doubles the accumulators; the two accumulator sets sit 256 columns apart
+// in tensor memory and the gate's accumulator 128 columns after the up projection's.  The host
+// picks the width per call (a multiple of 32) so that the tiles fill whole waves of SMs.
+constexpr int kTcMaxBN = 256;
+constexpr int kTcMaxBNGated = 128;
+constexpr uint32_t kTcAccStride = 256;     // tensor-memory columns between the two accumulator sets
+constexpr uint32_t kTcGateOfs = 128;       // columns between the two accumulators of a gated set
 constexpr int kTcBK = 64;                  // reduction slice per stage: 128 bytes of bf16 = one swizzle row
 constexpr int kTcUmmaK = 16;
 constexpr int kTcThreads = 192;            // warp 0 copies, warp 1 MMA + tensor memory, warps 2..5 epilogue
@@ -36,6 +41,7 @@ struct TcParams {
     uint32_t idesc;             // tcgen05 instruction descriptor (operand formats, tile shape)
     int stages;
     int tiles_m, tiles_n;
+    int bn;                     // neurons per tile
     long long ld_out;           // row stride of `out`, elements
     float* out;                 // [T][ld_out] fp32
     const void* bias;           // [N] in the input type, or NULL (not gated)
@@ -128,11 +134,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                   const __grid_constant__ CUtensorMap map_gate, const TcParams p)
 {
     constexpr int NB = GATED ? 2 : 1;                          // weight matrices per stage
-    constexpr int kTcBN = tc_bn(GATED);
-    constexpr uint32_t W_TILE_BYTES = (uint32_t)kTcBN * kTcBK * 2;     // one weight slice: kTcBN rows of 128 bytes
-    constexpr uint32_t STAGE_BYTES = kTcTileBytes + NB * W_TILE_BYTES;
-    constexpr uint32_t ACC_COLS = NB * kTcBN;                  // tensor-memory columns of one accumulator set
-    constexpr uint32_t TMEM_COLS = 2 * ACC_COLS;               // two sets: 512 columns
+    const int BN = p.bn;
+    const uint32_t W_TILE_BYTES = (uint32_t)BN * kTcBK * 2;    // one weight slice: BN rows of 128 bytes
+    const uint32_t STAGE_BYTES = kTcTileBytes + NB * W_TILE_BYTES;
+    constexpr uint32_t TMEM_COLS = 2 * kTcAccStride;           // two accumulator sets: all 512 columns
     const uint32_t IDESC = p.idesc;
 
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -177,7 +182,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
             uint32_t ph = 0;
             for (int tile = blockIdx.x; tile < n_tiles && !*abort_flag; tile += gridDim.x) {
                 // neighbouring CTAs share the weight slice (same tile_n), so it is read from HBM once
-                const int m0 = (tile % p.tiles_m) * kTcBM, n0 = (tile / p.tiles_m) * kTcBN;
+                const int m0 = (tile % p.tiles_m) * kTcBM, n0 = (tile / p.tiles_m) * BN;
                 for (int kb = 0; kb < kblocks; ++kb) {
                     if (!tc_wait(smem_u32(&empty_bar[s]), ph ^ 1u, abort_flag, p.status)) break;
                     const uint32_t fb = smem_u32(&full_bar[s]);
@@ -201,7 +206,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                 const uint32_t aph = (uint32_t)((it >> 1) & 1);
                 if (!tc_wait(smem_u32(&acc_empty[a]), aph ^ 1u, abort_flag, p.status)) break;
                 tc_fence_after();
-                const uint32_t d_up = tmem_base + (uint32_t)a * ACC_COLS;
+                const uint32_t d_up = tmem_base + (uint32_t)a * kTcAccStride;
                 bool ok = true;
                 for (int kb = 0; kb < kblocks; ++kb) {
                     if (!(ok = tc_wait(smem_u32(&full_bar[s]), ph, abort_flag, p.status))) break;
@@ -215,7 +220,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                         const uint32_t acc = (kb > 0 || k4 > 0) ? 1u : 0u;
                         const uint64_t koff = (uint64_t)(k4 * kTcUmmaK * 2 >> 4);       // 32 bytes per step, in 16-byte units
                         umma_bf16(d_up, da + koff, db + koff, IDESC, acc);
-                        if (GATED) umma_bf16(d_up + kTcBN, da + koff, dg + koff, IDESC, acc);
+                        if (GATED) umma_bf16(d_up + kTcGateOfs, da + koff, dg + koff, IDESC, acc);
                     }
                     umma_commit(smem_u32(&empty_bar[s]));       // the stage is free once these MMAs have read it
                     if (++s == p.stages) { s = 0; ph ^= 1u; }
@@ -232,17 +237,17 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
             if (*abort_flag) break;
             const int a = it & 1;
             const uint32_t aph = (uint32_t)((it >> 1) & 1);
-            const int m0 = (tile % p.tiles_m) * kTcBM, n0 = (tile / p.tiles_m) * kTcBN;
+            const int m0 = (tile % p.tiles_m) * kTcBM, n0 = (tile / p.tiles_m) * BN;
             if (!tc_wait(smem_u32(&acc_full[a]), aph, abort_flag, p.status)) break;
             tc_fence_after();
             const int row = m0 + q * 32 + lane;
-            const uint32_t t_up = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)a * ACC_COLS;
+            const uint32_t t_up = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)a * kTcAccStride;
             float* orow = p.out + (size_t)(row < p.T ? row : 0) * p.ld_out;
 #pragma unroll 1
-            for (int c = 0; c < kTcBN / 32; ++c) {
+            for (int c = 0; c < BN / 32; ++c) {
                 uint32_t u[32], g[32];
                 tmem_ld32(t_up + (uint32_t)(c * 32), u);
-                if (GATED) tmem_ld32(t_up + kTcBN + (uint32_t)(c * 32), g);
+                if (GATED) tmem_ld32(t_up + kTcGateOfs + (uint32_t)(c * 32), g);
                 tmem_ld_wait();
                 const int nbase = n0 + c * 32;
                 if (row < p.T) {
@@ -290,6 +295,26 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
     }
+}
+
+// Tile width for a call: the tiles run in waves of one per SM, a wave lasts about as long as its
+// width, so the width (a multiple of 32 up to the kind's maximum, at least half of it) with the
+// smallest waves x width wins; the wider one on a tie.
+static int tc_pick_bn(bool gated, int T, int N, int sms)
+{
+    const int max_bn = gated ? kTcMaxBNGated : kTcMaxBN;
+    const long long tiles_m = (T + kTcBM - 1) / kTcBM;
+    int best = max_bn;
+    long long best_cost = -1;
+    for (int bn = max_bn; bn >= max_bn / 2; bn -= 32) {
+        const long long tiles = tiles_m * ((N + bn - 1) / bn);
+        const long long cost = ((tiles + sms - 1) / sms) * bn;
+        if (best_cost < 0 || cost < best_cost) {
+            best_cost = cost;
+            best = bn;
+        }
+    }
+    return best;
 }
 
 // cuTensorMapEncodeTiled, looked up through the runtime (the library links no libcuda symbol).
@@ -366,10 +391,10 @@ coreinfer_status coreinfer_prefill_activations(const void* x, int32_t T, coreinf
     cudaStream_t st = (cudaStream_t)cuda_stream;
 
     CUtensorMap map_x, map_up, map_gate;
-    const int kTcBN = tc_bn(gated);
+    const int bn = tc_pick_bn(gated, T, d_ff, di.sm_count);
     if ((s = make_map(&map_x, x, T, d_model, f16, kTcBM)) != COREINFER_OK) return s;
-    if ((s = make_map(&map_up, w_up, d_ff, d_model, f16, kTcBN)) != COREINFER_OK) return s;
-    if ((s = make_map(&map_gate, gated ? w_gate : w_up, d_ff, d_model, f16, kTcBN)) != COREINFER_OK) return s;
+    if ((s = make_map(&map_up, w_up, d_ff, d_model, f16, bn)) != COREINFER_OK) return s;
+    if ((s = make_map(&map_gate, gated ? w_gate : w_up, d_ff, d_model, f16, bn)) != COREINFER_OK) return s;
 
     TcParams p;
     p.T = T;
@@ -381,14 +406,15 @@ coreinfer_status coreinfer_prefill_activations(const void* x, int32_t T, coreinf
     // instruction descriptor: fp32 accumulate (bit 4), A and B format (bits 7.. and 10..: 0 fp16, 1 bf16; one
     // instruction takes both operands in the same format), both K-major, N >> 3 at bit 17, M >> 4 at bit 24
     const uint32_t fmt = f16 ? 0u : 1u;
-    p.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(kTcBN >> 3) << 17) | ((uint32_t)(kTcBM >> 4) << 24);
+    p.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(kTcBM >> 4) << 24);
     p.tiles_m = (T + kTcBM - 1) / kTcBM;
-    p.tiles_n = (d_ff + kTcBN - 1) / kTcBN;
+    p.tiles_n = (d_ff + bn - 1) / bn;
+    p.bn = bn;
     p.ld_out = ld_act;
     p.out = act_out;
     p.bias = b_up;
     p.status = (unsigned*)workspace;
-    const size_t stage = (size_t)kTcTileBytes + (size_t)(gated ? 2 : 1) * kTcBN * kTcBK * 2;
+    const size_t stage = (size_t)kTcTileBytes + (size_t)(gated ? 2 : 1) * bn * kTcBK * 2;
     const size_t fixed = 1024 /* alignment slack */ + (2 * kTcMaxStages + 4) * sizeof(uint64_t) + 64;
     long long stages = ((long long)di.smem_optin - (long long)fixed) / (long long)stage;
     if (stages > kTcMaxStages) stages = kTcMaxStages;

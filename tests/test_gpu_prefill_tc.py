@@ -75,3 +75,24 @@ def test_full_size_layer_and_selection_on_its_output(name):
     S_o, f_o = oracle.select(A.cpu().numpy(), cfg.alpha, cfg.beta)
     np.testing.assert_array_equal(f, f_o)
     np.testing.assert_array_equal(S, S_o)
+
+
+@pytest.mark.parametrize("gated,width", [(False, 256), (False, 224), (False, 192), (False, 160), (True, 96), (True, 64)])
+def test_every_tile_width_the_host_can_pick(gated, width):
+    """The tile width is picked per call so that the tiles fill whole waves of the GPU's SMs:
+    with one row tile and d_ff = (SM count) x width - 4 exactly that width wins (every wider one
+    needs as many waves for wider tiles, the next narrower one a second wave), and the last tile
+    of the ragged d_ff is cut.  Integer inputs: bit-exact against the oracle on all rows."""
+    require_gpu()
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    T, d, N = 100, 192, sms * width - 4
+    rng = np.random.default_rng(width)
+    mk = lambda *s: torch.from_numpy(rng.integers(-3, 4, size=s).astype(np.float32)).to(torch.bfloat16).cuda()
+    X, w_up = mk(T, d), mk(N, d)
+    w_gate = mk(N, d) if gated else None
+    b_up = None if gated else mk(N)
+    kind = ci.FFN_RELU_GATED if gated else ci.FFN_RELU
+    A = _tc(X, kind, w_up, w_gate, b_up).cpu().numpy()
+    H_o, _ = oracle.ffn_dense(to_f32_np(X), kind, to_f32_np(w_up), to_f32_np(w_gate), np.zeros((d, N), np.float32),
+                              to_f32_np(b_up), None, want_y=False)
+    np.testing.assert_array_equal(A, H_o)
