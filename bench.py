@@ -630,6 +630,17 @@ def extension_times(ci, wl, peak):
     gi = torch.empty(1, dtype=torch.int32, device="cuda")
     out["nearest_centroid_16_groups_us"] = 1e3 * _time_ms(lambda: ci.coreinfer_nearest_centroid(C, v, gi, cws, stream), stream, 20)
     w_up, _, w_down = wl.layer_weights(c2, 0, device="cuda")
+    # activations kept in bf16: tensor-core pre-fill writing bf16, selection reading it
+    X = wl.prompt_hidden(c2, device="cuda")
+    A16 = torch.empty((c2.T, N), dtype=torch.bfloat16, device="cuda")
+    tws = torch.empty(ci.coreinfer_prefill_activations_workspace_bytes(), dtype=torch.uint8, device="cuda")
+    sws = torch.empty(ci.coreinfer_select_workspace_bytes(c2.T, N), dtype=torch.uint8, device="cuda")
+    out["activations_bf16_out_us"] = 1e3 * _time_ms(
+        lambda: ci.coreinfer_prefill_activations(X, ci.FFN_RELU, w_up, None, None, A16, tws, stream), stream, 10)
+    out["select_on_bf16_us"] = 1e3 * _time_ms(
+        lambda: ci.coreinfer_select_core(A16, c2.alpha, c2.beta, S, None, sws, stream), stream, 10)
+    ci.coreinfer_workspace_status(tws)
+    ci.coreinfer_workspace_status(sws)
     new = lambda: torch.empty((K2, c2.d_model), dtype=c2.torch_dtype, device="cuda")
     up_c, down_c = new(), new()
     ci.coreinfer_compact(w_up, None, w_down, None, a, K2, up_c, None, down_c, None, stream)

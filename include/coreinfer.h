@@ -86,8 +86,10 @@ const char* coreinfer_last_error(void);
  * is the K = coreinfer_count(beta, d_ff) neurons with the largest f (equal
  * counts go to the lower index), written in ascending index order.
  *
- *   act         device, [T, d_ff] with row stride ld_act elements; fp32
- *               (COREINFER_F32 only).  ld_act >= d_ff, ld_act % 4 == 0.
+ *   act         device, [T, d_ff] with row stride ld_act elements; fp32 (the precision the
+ *               method keeps activations in), bf16 or fp16 (widened exactly: order, sign, zero
+ *               and NaN are those of the stored values).  ld_act >= d_ff and a multiple of 4
+ *               (fp32) or 8 (16-bit): every row starts on a 16-byte boundary.
  *   core_idx    device, out, K int32 (capacity >= K).
  *   counts_out  device, out, [d_ff] int32 = f, or NULL.
  *   workspace   device scratch of at least coreinfer_select_workspace_bytes();
@@ -352,14 +354,17 @@ coreinfer_status coreinfer_update_core_set(const void* w_up, const void* w_gate,
  * applied to, produced the way the method obtains it -- as the intermediate result of the dense
  * pre-fill pass (Section 4.2, Fig. 1) -- without the down projection:
  *   RELU:        A = max(X W_up^T + b_up, 0)        RELU_GATED:  A = max(X W_gate^T, 0) * (X W_up^T)
- * bf16 inputs, exact products, fp32 accumulation (tcgen05.mma into tensor memory), fp32 output.
+ * bf16 or fp16 inputs, exact products, fp32 accumulation (tcgen05.mma into tensor memory); the
+ * output is fp32 (the precision the method keeps activations in, Section 5 "Models") or, rounded
+ * to nearest even once after the activation, bf16 / fp16 for half the bytes.
  * The summation order differs from coreinfer_ffn_dense_ref's, so the two agree to fp32 rounding
  * (1e-4 relative), not bit for bit; selection is exact on whichever tensor it is given.
  *
  *   x        device [T, d_model] bf16            w_up   device [d_ff, d_model] bf16
  *   w_gate   device [d_ff, d_model] bf16 or NULL (NULL iff RELU)
  *   b_up     device [d_ff] bf16 or NULL (RELU only)
- *   act_out  device out [T, d_ff] fp32 with row stride ld_act elements (ld_act >= d_ff, % 4 == 0)
+ *   act_out  device out [T, d_ff] of act_dtype with row stride ld_act elements (ld_act >= d_ff and a
+ *            multiple of 4 for fp32, of 8 for bf16 / fp16: the layout coreinfer_select_core takes)
  *   workspace  device, at least coreinfer_prefill_activations_workspace_bytes(); its first word is
  *              a status word readable with coreinfer_workspace_status.
  * d_model must be a multiple of 8.  Any T and d_ff (edges are zero-filled and masked).
@@ -369,7 +374,7 @@ size_t coreinfer_prefill_activations_workspace_bytes(void);
 coreinfer_status coreinfer_prefill_activations(const void* x, int32_t T, coreinfer_dtype dtype,
                                                coreinfer_ffn_kind kind, int32_t d_model, int32_t d_ff,
                                                const void* w_up, const void* w_gate, const void* b_up,
-                                               float* act_out, int64_t ld_act,
+                                               void* act_out, coreinfer_dtype act_dtype, int64_t ld_act,
                                                void* workspace, size_t workspace_bytes,
                                                void* cuda_stream);
 

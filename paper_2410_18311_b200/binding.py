@@ -111,7 +111,7 @@ def load() -> ctypes.CDLL:
     lib.coreinfer_prefill_activations_workspace_bytes.restype = sz
     lib.coreinfer_prefill_activations_workspace_bytes.argtypes = []
     lib.coreinfer_prefill_activations.restype = ctypes.c_int
-    lib.coreinfer_prefill_activations.argtypes = [vp, i32, ctypes.c_int, ctypes.c_int, i32, i32, vp, vp, vp, vp, i64,
+    lib.coreinfer_prefill_activations.argtypes = [vp, i32, ctypes.c_int, ctypes.c_int, i32, i32, vp, vp, vp, vp, ctypes.c_int, i64,
                                                   vp, sz, vp]
     lib.coreinfer_counts_add.restype = ctypes.c_int
     lib.coreinfer_counts_add.argtypes = [vp, vp, i32, vp]
@@ -172,7 +172,7 @@ def coreinfer_select_workspace_bytes(T: int, d_ff: int) -> int:
 
 def coreinfer_select_core(act, alpha, beta, core_idx, counts_out, workspace, stream=None,
                           T=None, d_ff=None, ld_act=None, act_dtype=None):
-    """act [T, d_ff] fp32 (row stride ld_act) -> core_idx [K] int32 ascending, counts_out [d_ff] | None."""
+    """act [T, d_ff] fp32, bf16 or fp16 (row stride ld_act) -> core_idx [K] int32 ascending, counts_out [d_ff] | None."""
     T = act.shape[0] if T is None else T
     d_ff = act.shape[1] if d_ff is None else d_ff
     ld_act = act.stride(0) if ld_act is None else ld_act
@@ -273,11 +273,11 @@ def coreinfer_prefill_activations_workspace_bytes() -> int:
 
 
 def coreinfer_prefill_activations(x, kind, w_up, w_gate, b_up, act_out, workspace, stream=None):
-    """x [T, d] bf16, w_up / w_gate [d_ff, d] bf16 -> act_out [T, d_ff] fp32 (tensor cores)."""
+    """x [T, d], w_up / w_gate [d_ff, d] bf16 or fp16 -> act_out [T, d_ff] fp32, bf16 or fp16 (tensor cores)."""
     T, d_model = x.shape
     d_ff = w_up.shape[0]
     _check(load().coreinfer_prefill_activations(_p(x), T, dtype_code(x), int(kind), d_model, d_ff, _p(w_up), _p(w_gate),
-                                                _p(b_up), _p(act_out), act_out.stride(0), _p(workspace),
+                                                _p(b_up), _p(act_out), dtype_code(act_out), act_out.stride(0), _p(workspace),
                                                 workspace.numel() * workspace.element_size(), _stream(stream)))
 
 

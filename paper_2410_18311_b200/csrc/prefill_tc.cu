@@ -43,7 +43,8 @@ struct TcParams {
     int tiles_m, tiles_n;
     int bn;                     // neurons per tile
     long long ld_out;           // row stride of `out`, elements
-    float* out;                 // [T][ld_out] fp32
+    void* out;                  // [T][ld_out] in the output type
+    int out_kind;               // 0 fp32, 1 bf16, 2 fp16 (rounded to nearest even once, after the activation)
     const void* bias;           // [N] in the input type, or NULL (not gated)
     int f16;                    // inputs are fp16 (else bf16)
     unsigned* status;
@@ -242,7 +243,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
             tc_fence_after();
             const int row = m0 + q * 32 + lane;
             const uint32_t t_up = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)a * kTcAccStride;
-            float* orow = p.out + (size_t)(row < p.T ? row : 0) * p.ld_out;
+            const size_t orow_ofs = (size_t)(row < p.T ? row : 0) * p.ld_out;
+            float* orow = reinterpret_cast<float*>(p.out) + orow_ofs;
+            uint16_t* orow16 = reinterpret_cast<uint16_t*>(p.out) + orow_ofs;
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
                 uint32_t u[32], g[32];
@@ -266,12 +269,28 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                                 v[e] = fmaxf(uu, 0.f);
                             }
                         }
-                        if (nbase + j + 3 < p.N) {
-                            *reinterpret_cast<float4*>(orow + nbase + j) = make_float4(v[0], v[1], v[2], v[3]);
+                        if (p.out_kind == 0) {
+                            if (nbase + j + 3 < p.N) {
+                                *reinterpret_cast<float4*>(orow + nbase + j) = make_float4(v[0], v[1], v[2], v[3]);
+                            } else {
+#pragma unroll
+                                for (int e = 0; e < 4; ++e)
+                                    if (nbase + j + e < p.N) orow[nbase + j + e] = v[e];
+                            }
                         } else {
+                            uint16_t h[4];
 #pragma unroll
                             for (int e = 0; e < 4; ++e)
-                                if (nbase + j + e < p.N) orow[nbase + j + e] = v[e];
+                                h[e] = p.out_kind == 1 ? __bfloat16_as_ushort(__float2bfloat16_rn(v[e]))
+                                                       : __half_as_ushort(__float2half_rn(v[e]));
+                            if (nbase + j + 3 < p.N) {
+                                *reinterpret_cast<uint2*>(orow16 + nbase + j) =
+                                    make_uint2((uint32_t)h[0] | ((uint32_t)h[1] << 16), (uint32_t)h[2] | ((uint32_t)h[3] << 16));
+                            } else {
+#pragma unroll
+                                for (int e = 0; e < 4; ++e)
+                                    if (nbase + j + e < p.N) orow16[nbase + j + e] = h[e];
+                            }
                         }
                     }
                 }
@@ -364,8 +383,8 @@ size_t coreinfer_prefill_activations_workspace_bytes(void) { return 256; }
 
 coreinfer_status coreinfer_prefill_activations(const void* x, int32_t T, coreinfer_dtype dtype, coreinfer_ffn_kind kind,
                                                int32_t d_model, int32_t d_ff, const void* w_up, const void* w_gate,
-                                               const void* b_up, float* act_out, int64_t ld_act, void* workspace,
-                                               size_t workspace_bytes, void* cuda_stream)
+                                               const void* b_up, void* act_out, coreinfer_dtype act_dtype, int64_t ld_act,
+                                               void* workspace, size_t workspace_bytes, void* cuda_stream)
 {
     if (dtype != COREINFER_BF16 && dtype != COREINFER_F16)
         CI_FAIL(COREINFER_ERR_UNSUPPORTED, "the tensor-core pre-fill takes bf16 or fp16 inputs (dtype %d given); "
@@ -380,7 +399,10 @@ coreinfer_status coreinfer_prefill_activations(const void* x, int32_t T, coreinf
     if (gated != (w_gate != nullptr) || (w_gate && !aligned16(w_gate)))
         CI_FAIL(COREINFER_ERR_INVALID_ARG, "w_gate must be given (16-byte aligned) exactly for the gated FFN");
     if (gated && b_up) CI_FAIL(COREINFER_ERR_INVALID_ARG, "the gated FFN has no up bias");
-    if (ld_act < d_ff || (ld_act & 3) != 0) CI_FAIL(COREINFER_ERR_INVALID_ARG, "ld_act must be >= d_ff and a multiple of 4");
+    if (!dtype_known(act_dtype)) CI_FAIL(COREINFER_ERR_UNSUPPORTED, "act_dtype %d is not supported", (int)act_dtype);
+    const int act_per16 = 16 / (int)dtype_size(act_dtype);
+    if (ld_act < d_ff || (ld_act % act_per16) != 0)
+        CI_FAIL(COREINFER_ERR_INVALID_ARG, "ld_act must be >= d_ff and a multiple of %d (rows of whole 16-byte pieces)", act_per16);
     if (!workspace || !aligned16(workspace)) CI_FAIL(COREINFER_ERR_WORKSPACE, "workspace is NULL or misaligned");
     if (workspace_bytes < coreinfer_prefill_activations_workspace_bytes())
         CI_FAIL(COREINFER_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes,
@@ -412,6 +434,7 @@ coreinfer_status coreinfer_prefill_activations(const void* x, int32_t T, coreinf
     p.bn = bn;
     p.ld_out = ld_act;
     p.out = act_out;
+    p.out_kind = act_dtype == COREINFER_F32 ? 0 : (act_dtype == COREINFER_BF16 ? 1 : 2);
     p.bias = b_up;
     p.status = (unsigned*)workspace;
     const size_t stage = (size_t)kTcTileBytes + (size_t)(gated ? 2 : 1) * bn * kTcBK * 2;

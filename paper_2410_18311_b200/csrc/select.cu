@@ -42,6 +42,23 @@ __device__ __forceinline__ int count_dev(double frac, int n)
 
 __device__ __forceinline__ bool is_pos_bits(uint32_t b) { return (b - 1u) < 0x7F800000u; }
 
+// The fp32 bit patterns of the four entries of group v of a row in shared memory.  16-bit
+// inputs widen exactly (bf16: its bits are the upper half of the fp32 pattern; fp16: every
+// value, subnormals included, is an fp32 value), so order, sign, zero and NaN are those of the
+// stored values.  in_kind: 0 fp32, 1 bf16, 2 fp16.
+__device__ __forceinline__ uint32_t half_to_f32_bits(uint32_t h)
+{
+    return __float_as_uint(__half2float(__ushort_as_half((unsigned short)h)));
+}
+__device__ __forceinline__ uint4 load_group(const uint8_t* row, int v, int in_kind)
+{
+    if (in_kind == 0) return reinterpret_cast<const uint4*>(row)[v];
+    const uint2 w = reinterpret_cast<const uint2*>(row)[v];
+    if (in_kind == 1) return make_uint4(w.x << 16, w.x & 0xffff0000u, w.y << 16, w.y & 0xffff0000u);
+    return make_uint4(half_to_f32_bits(w.x & 0xffffu), half_to_f32_bits(w.x >> 16),
+                      half_to_f32_bits(w.y & 0xffffu), half_to_f32_bits(w.y >> 16));
+}
+
 struct SelShared {
     int warp_tot[kSelWarps];
     int bin, above, bin_count, total;
@@ -107,7 +124,7 @@ __device__ __forceinline__ int find_bin(const int* hist, int k, bool k_from_tota
 // free for the next row at once); otherwise every pass re-reads them from shared memory.
 template <int VPT, bool HOLD>
 __global__ void __launch_bounds__(kSelThreads, 1)
-select_rows_kernel(const float* __restrict__ act, int T, int N, long long ld, double alpha,
+select_rows_kernel(const uint8_t* __restrict__ act, int T, int N, long long ld_bytes, int in_kind, double alpha,
                    uint16_t* __restrict__ partial, unsigned* __restrict__ status, int nbuf, int row_bytes)
 {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -118,7 +135,7 @@ select_rows_kernel(const float* __restrict__ act, int T, int N, long long ld, do
 
     const int tid = threadIdx.x;
     const int G = gridDim.x;
-    const int nvec = row_bytes / 16;
+    const int nvec = (N + 3) >> 2;         // groups of four entries
 
     if (tid == 0) {
         mbar_init(smem_u32(&bars[0]), 1);
@@ -132,7 +149,7 @@ select_rows_kernel(const float* __restrict__ act, int T, int N, long long ld, do
     auto issue_row = [&](int t, int b) {   // thread 0 only
         const uint32_t bar = smem_u32(&bars[b]);
         mbar_arrive_expect_tx(bar, (uint32_t)row_bytes);
-        const uint8_t* src = reinterpret_cast<const uint8_t*>(act + (long long)t * ld);
+        const uint8_t* src = act + (long long)t * ld_bytes;
         const uint32_t dst = smem_u32(smem + (size_t)b * buf_bytes);
         for (uint32_t off = 0; off < (uint32_t)row_bytes; off += kCopyChunk) {
             const uint32_t n = min(kCopyChunk, (uint32_t)row_bytes - off);
@@ -175,12 +192,12 @@ select_rows_kernel(const float* __restrict__ act, int T, int N, long long ld, do
         __syncthreads();
         if (sh->abort_flag) break;   // block-uniform
 
-        const uint4* row = reinterpret_cast<const uint4*>(smem + (size_t)b * buf_bytes);
+        const uint8_t* row = smem + (size_t)b * buf_bytes;
         // masked bit patterns of vector i: 0 stands for "not positive" (or beyond d_ff)
         auto load_vec = [&](int i) -> uint4 {
             const int v = tid + i * kSelThreads;
             uint4 q = make_uint4(0, 0, 0, 0);
-            if (v < nvec) q = row[v];
+            if (v < nvec) q = load_group(row, v, in_kind);
             if (v * 4 + 0 >= N || !is_pos_bits(q.x)) q.x = 0u;
             if (v * 4 + 1 >= N || !is_pos_bits(q.y)) q.y = 0u;
             if (v * 4 + 2 >= N || !is_pos_bits(q.z)) q.z = 0u;
@@ -300,7 +317,7 @@ constexpr int kWarpHistStride = 288;     // 256 exponent bins + 32 words (one pe
 
 template <int VPT>
 __global__ void __launch_bounds__(kSelThreads, 1)
-select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long ld, double alpha,
+select_rows_fast_kernel(const uint8_t* __restrict__ act, int T, int N, long long ld_bytes, int in_kind, double alpha,
                         uint16_t* __restrict__ partial, unsigned* __restrict__ status, int row_bytes)
 {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -312,7 +329,7 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
 
     const int tid = threadIdx.x;
     const int G = gridDim.x;
-    const int nvec = row_bytes / 16;
+    const int nvec = (N + 3) >> 2;         // groups of four entries
 
     if (tid == 0) {
         mbar_init(smem_u32(bar), 1);
@@ -327,7 +344,7 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
     auto issue_row = [&](int t) {          // thread 0 only
         const uint32_t b = smem_u32(bar);
         mbar_arrive_expect_tx(b, (uint32_t)row_bytes);
-        const uint8_t* src = reinterpret_cast<const uint8_t*>(act + (long long)t * ld);
+        const uint8_t* src = act + (long long)t * ld_bytes;
         const uint32_t dst = smem_u32(smem);
         for (uint32_t off = 0; off < (uint32_t)row_bytes; off += kCopyChunk) {
             const uint32_t n = min(kCopyChunk, (uint32_t)row_bytes - off);
@@ -366,13 +383,13 @@ select_rows_fast_kernel(const float* __restrict__ act, int T, int N, long long l
         // as a signed integer and far from all of them as an unsigned difference, so no loop below
         // needs a test for it.
         constexpr uint32_t kMasked = 0x80000000u;
-        const uint4* row = reinterpret_cast<const uint4*>(smem);
+        const uint8_t* row = smem;
         uint4 held[VPT];
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
             const int v = tid + i * kSelThreads;
             uint4 q = make_uint4(0, 0, 0, 0);
-            if (v < nvec) q = row[v];
+            if (v < nvec) q = load_group(row, v, in_kind);
             q.x = is_pos_bits(q.x) ? q.x : kMasked;
             q.y = is_pos_bits(q.y) ? q.y : kMasked;
             q.z = is_pos_bits(q.z) ? q.z : kMasked;
@@ -642,13 +659,13 @@ select_top_kernel(const int32_t* __restrict__ f, int N, int K, int T, int32_t* _
 static size_t sel_fixed_smem() { return kSelBins * sizeof(int) + 2 * sizeof(uint64_t) + sizeof(SelShared) + 128; }
 
 template <int VPT>
-static coreinfer_status launch_rows(int grid, size_t smem, cudaStream_t st, const float* act, int T, int N,
-                                    long long ld, double alpha, uint16_t* partial, unsigned* status, int nbuf,
-                                    int row_bytes)
+static coreinfer_status launch_rows(int grid, size_t smem, cudaStream_t st, const uint8_t* act, int T, int N,
+                                    long long ld_bytes, int in_kind, double alpha, uint16_t* partial,
+                                    unsigned* status, int nbuf, int row_bytes)
 {
     auto kern = select_rows_kernel<VPT, (VPT <= 5)>;
     CI_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    kern<<<grid, kSelThreads, smem, st>>>(act, T, N, ld, alpha, partial, status, nbuf, row_bytes);
+    kern<<<grid, kSelThreads, smem, st>>>(act, T, N, ld_bytes, in_kind, alpha, partial, status, nbuf, row_bytes);
     CI_CUDA(cudaGetLastError());
     return COREINFER_OK;
 }
@@ -660,13 +677,13 @@ static size_t sel_fast_fixed_smem()
 }
 
 template <int VPT>
-static coreinfer_status launch_rows_fast(int grid, size_t smem, cudaStream_t st, const float* act, int T, int N,
-                                         long long ld, double alpha, uint16_t* partial, unsigned* status,
-                                         int row_bytes)
+static coreinfer_status launch_rows_fast(int grid, size_t smem, cudaStream_t st, const uint8_t* act, int T, int N,
+                                         long long ld_bytes, int in_kind, double alpha, uint16_t* partial,
+                                         unsigned* status, int row_bytes)
 {
     auto kern = select_rows_fast_kernel<VPT>;
     CI_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    kern<<<grid, kSelThreads, smem, st>>>(act, T, N, ld, alpha, partial, status, row_bytes);
+    kern<<<grid, kSelThreads, smem, st>>>(act, T, N, ld_bytes, in_kind, alpha, partial, status, row_bytes);
     CI_CUDA(cudaGetLastError());
     return COREINFER_OK;
 }
@@ -711,16 +728,19 @@ coreinfer_status coreinfer_select_core(const void* act, coreinfer_dtype act_dtyp
                                        int32_t* counts_out, void* workspace, size_t workspace_bytes,
                                        void* cuda_stream)
 {
-    if (act_dtype != COREINFER_F32)
-        CI_FAIL(COREINFER_ERR_UNSUPPORTED, "activations must be fp32 (dtype %d given)", (int)act_dtype);
+    if (!dtype_known(act_dtype))
+        CI_FAIL(COREINFER_ERR_UNSUPPORTED, "activations must be fp32, bf16 or fp16 (dtype %d given)", (int)act_dtype);
+    const int esize = (int)dtype_size(act_dtype);
+    const int in_kind = act_dtype == COREINFER_F32 ? 0 : (act_dtype == COREINFER_BF16 ? 1 : 2);
+    const int per16 = 16 / esize;          // entries per 16 bytes: rows start and end on 16-byte boundaries
     if (!act || !core_idx) CI_FAIL(COREINFER_ERR_INVALID_ARG, "act / core_idx is NULL");
     if (T < 1 || d_ff < 1) CI_FAIL(COREINFER_ERR_INVALID_ARG, "T = %d, d_ff = %d must be >= 1", T, d_ff);
     if (!(alpha > 0.0 && alpha <= 1.0) || !(beta > 0.0 && beta <= 1.0))
         CI_FAIL(COREINFER_ERR_INVALID_ARG, "alpha = %g, beta = %g must lie in (0, 1]", alpha, beta);
     if (coreinfer_count(beta, d_ff) < 1)
         CI_FAIL(COREINFER_ERR_INVALID_ARG, "beta = %g selects no neuron of d_ff = %d", beta, d_ff);
-    if (ld_act < d_ff || (ld_act & 3) != 0 || !aligned16(act))
-        CI_FAIL(COREINFER_ERR_INVALID_ARG, "act must be 16-byte aligned with ld_act >= d_ff and ld_act %% 4 == 0");
+    if (ld_act < d_ff || (ld_act % per16) != 0 || !aligned16(act))
+        CI_FAIL(COREINFER_ERR_INVALID_ARG, "act must be 16-byte aligned with ld_act >= d_ff and ld_act %% %d == 0", per16);
     if (d_ff > kSelMaxVpt * kSelThreads * 4)
         CI_FAIL(COREINFER_ERR_UNSUPPORTED, "d_ff = %d exceeds %d", d_ff, kSelMaxVpt * kSelThreads * 4);
     if (!workspace || !aligned16(workspace)) CI_FAIL(COREINFER_ERR_WORKSPACE, "workspace is NULL or misaligned");
@@ -733,7 +753,7 @@ coreinfer_status coreinfer_select_core(const void* act, coreinfer_dtype act_dtyp
     cudaStream_t st = (cudaStream_t)cuda_stream;
 
     const int n4 = (d_ff + 3) & ~3;
-    const int row_bytes = n4 * 4;
+    const int row_bytes = (d_ff + per16 - 1) / per16 * 16;       // whole 16-byte pieces, within ld_act entries
     int G = T < di.sm_count ? T : di.sm_count;
     if (G > kSelMaxCtas) G = kSelMaxCtas;
     const size_t buf = ((size_t)row_bytes + 127) & ~(size_t)127;
@@ -760,10 +780,11 @@ coreinfer_status coreinfer_select_core(const void* act, coreinfer_dtype act_dtyp
     const int vpt = (n4 / 4 + kSelThreads - 1) / kSelThreads;
 #define CI_ROWS(V)                                                                                        \
     case V:                                                                                               \
-        s = fast ? launch_rows_fast<V>(G, smem_fast, st, (const float*)act, T, d_ff, (long long)ld_act,   \
-                                       alpha, partial, status, row_bytes)                                 \
-                 : launch_rows<V>(G, smem, st, (const float*)act, T, d_ff, (long long)ld_act, alpha,      \
-                                  partial, status, nbuf, row_bytes);                                      \
+        s = fast ? launch_rows_fast<V>(G, smem_fast, st, (const uint8_t*)act, T, d_ff,                   \
+                                       (long long)ld_act * esize, in_kind, alpha, partial, status,        \
+                                       row_bytes)                                                         \
+                 : launch_rows<V>(G, smem, st, (const uint8_t*)act, T, d_ff, (long long)ld_act * esize,   \
+                                  in_kind, alpha, partial, status, nbuf, row_bytes);                      \
         break;
     switch (vpt) {
         CI_ROWS(1) CI_ROWS(2) CI_ROWS(3) CI_ROWS(4) CI_ROWS(5) CI_ROWS(6) CI_ROWS(7) CI_ROWS(8) CI_ROWS(9)

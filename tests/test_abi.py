@@ -44,7 +44,10 @@ def test_argument_errors_are_reported_without_a_device(lib):
     assert lib.coreinfer_select_core(null, ci.F32, 4, 8, 8, 0.4, 0.2, p, null, p, 1024, null) == ci.ERR_INVALID_ARG
     assert b"NULL" in lib.coreinfer_last_error()
     assert lib.coreinfer_select_core(p, ci.F32, 4, 8, 8, 1.5, 0.2, p, null, p, 1024, null) == ci.ERR_INVALID_ARG
-    assert lib.coreinfer_select_core(p, ci.BF16, 4, 8, 8, 0.4, 0.2, p, null, p, 1024, null) == ci.ERR_UNSUPPORTED
+    assert lib.coreinfer_select_core(p, 7, 4, 8, 8, 0.4, 0.2, p, null, p, 1024, null) == ci.ERR_UNSUPPORTED
+    # 16-bit rows must start on 16-byte boundaries: a row stride of 12 entries does for fp32, not for bf16
+    assert lib.coreinfer_select_core(p, ci.F32, 4, 8, 12, 0.4, 0.2, p, null, p, 16, null) == ci.ERR_WORKSPACE
+    assert lib.coreinfer_select_core(p, ci.BF16, 4, 8, 12, 0.4, 0.2, p, null, p, 1024, null) == ci.ERR_INVALID_ARG
     # a fraction inside (0, 1] that still rounds to an empty set
     assert lib.coreinfer_select_core(p, ci.F32, 4, 8, 8, 0.4, 1e-9, p, null, p, 1024, null) == ci.ERR_INVALID_ARG
     assert b"no neuron" in lib.coreinfer_last_error()

@@ -96,3 +96,50 @@ def test_every_tile_width_the_host_can_pick(gated, width):
     H_o, _ = oracle.ffn_dense(to_f32_np(X), kind, to_f32_np(w_up), to_f32_np(w_gate), np.zeros((d, N), np.float32),
                               to_f32_np(b_up), None, want_y=False)
     np.testing.assert_array_equal(A, H_o)
+
+
+@pytest.mark.parametrize("out_dtype", [torch.bfloat16, torch.float16])
+@pytest.mark.parametrize("gated", [False, True])
+def test_sixteen_bit_output_and_selection_on_it(out_dtype, gated):
+    """The activations written as bf16 / fp16 (one rounding after the activation; half the bytes):
+    integer inputs give the exactly rounded tensor; a full-width ragged layer stays within the
+    16-bit tolerance of the oracle and the selection on the stored values is bit-exact."""
+    require_gpu()
+    rng = np.random.default_rng(11)
+    T, d, N = 150, 256, 1004
+    mk = lambda *s: torch.from_numpy(rng.integers(-4, 5, size=s).astype(np.float32)).to(torch.bfloat16).cuda()
+    X, w_up = mk(T, d), mk(N, d)
+    w_gate = mk(N, d) if gated else None
+    kind = ci.FFN_RELU_GATED if gated else ci.FFN_RELU
+    ld = (N + 7) // 8 * 8
+    buf = torch.full((T, ld), float("nan"), dtype=out_dtype, device="cuda")
+    A = buf[:, :N]
+    ws = torch.empty(ci.coreinfer_prefill_activations_workspace_bytes(), dtype=torch.uint8, device="cuda")
+    ci.coreinfer_prefill_activations(X, kind, w_up, w_gate, None, A, ws)
+    ci.coreinfer_workspace_status(ws)
+    H_o, _ = oracle.ffn_dense(to_f32_np(X), kind, to_f32_np(w_up), to_f32_np(w_gate), np.zeros((d, N), np.float32),
+                              want_y=False)
+    expect = torch.from_numpy(H_o).to(out_dtype).to(torch.float32).numpy()     # round to nearest even, once
+    got = A.to(torch.float32).cpu().numpy()
+    np.testing.assert_array_equal(got, expect)
+    assert torch.isnan(buf[:, N:].float()).all()                              # the padding is not written
+
+    g = torch.Generator().manual_seed(5)
+    mkr = lambda *s, std=1.0: (torch.randn(*s, generator=g) * std).to(torch.bfloat16).cuda()
+    T, d, N = 260, 512, 3000
+    X, w_up = mkr(T, d), mkr(N, d, std=0.05)
+    w_gate = mkr(N, d, std=0.05) if gated else None
+    A = torch.empty((T, N), dtype=out_dtype, device="cuda")
+    ci.coreinfer_prefill_activations(X, kind, w_up, w_gate, None, A, ws)
+    ci.coreinfer_workspace_status(ws)
+    H_o, _ = oracle.ffn_dense(to_f32_np(X), kind, to_f32_np(w_up), to_f32_np(w_gate), np.zeros((d, N), np.float32),
+                              want_y=False)
+    A32 = A.to(torch.float32).cpu().numpy()
+    # one rounding of an fp32 result that itself is within 1e-4 (relative to the RMS) of the oracle's
+    rms = float(np.sqrt(np.mean(H_o.astype(np.float64) ** 2)))
+    bound = 0.5 * torch.finfo(out_dtype).eps * np.abs(H_o) * 1.001 + 2e-4 * rms
+    assert (np.abs(A32 - H_o) <= bound).all()
+    S, f = gpu_select(A, 0.4, 0.2)
+    S_o, f_o = oracle.select(A32, 0.4, 0.2)
+    np.testing.assert_array_equal(f, f_o)
+    np.testing.assert_array_equal(S, S_o)

@@ -151,3 +151,75 @@ def test_same_input_same_output_twice():
     S2, f2 = gpu_select(A, 0.4, 0.2)
     np.testing.assert_array_equal(S1, S2)
     np.testing.assert_array_equal(f1, f2)
+
+
+def _sixteen_bit(A32, dtype, ld_mult=8, fill=7.0):
+    """A [T, N] tensor of a 16-bit type inside a buffer whose rows are padded (with positive
+    garbage) to a multiple of 8 entries; returns the CUDA view and the values widened to fp32."""
+    T, N = A32.shape
+    ld = (N + ld_mult - 1) // ld_mult * ld_mult
+    buf = torch.full((T, ld), fill, dtype=dtype)
+    buf[:, :N] = torch.from_numpy(A32).to(dtype)
+    dev = buf.cuda()
+    return dev[:, :N], buf[:, :N].to(torch.float32).numpy()
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16])
+@pytest.mark.parametrize("T,N,alpha,beta", [
+    (1, 4, 0.4, 0.2), (3, 9, 0.5, 0.5), (7, 261, 0.4, 0.2), (33, 1003, 0.4, 0.25), (64, 3072, 0.4, 0.2),
+    (300, 4096 + 6, 0.4, 0.2), (20, 11008, 0.4, 0.25), (6, 36864, 0.4, 0.2), (4, 24581, 0.4, 0.2),
+])
+def test_sixteen_bit_activations(dtype, T, N, alpha, beta):
+    """bf16 / fp16 activations are ranked as the values they store: the sets and counts equal the
+    oracle's on the same values widened to fp32.  Sixteen-bit values tie often (a few hundred
+    distinct values per row), so the lower-index rule decides most thresholds."""
+    require_gpu()
+    rng = np.random.default_rng(T * 31 + N)
+    A = rng.standard_normal((T, N)).astype(np.float32)
+    A[rng.random((T, N)) < 0.2] = 0.0
+    view, A16 = _sixteen_bit(A, dtype)
+    S_o, f_o = oracle.select(A16, alpha, beta)
+    K = ci.coreinfer_count(beta, N)
+    S = torch.full((K,), -1, dtype=torch.int32, device="cuda")
+    f = torch.full((N,), -1, dtype=torch.int32, device="cuda")
+    ws = torch.empty(ci.coreinfer_select_workspace_bytes(T, N), dtype=torch.uint8, device="cuda")
+    ci.coreinfer_select_core(view, alpha, beta, S, f, ws, T=T, d_ff=N, ld_act=view.stride(0))
+    ci.coreinfer_workspace_status(ws)
+    np.testing.assert_array_equal(f.cpu().numpy(), f_o)
+    np.testing.assert_array_equal(S.cpu().numpy(), S_o)
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16])
+def test_sixteen_bit_special_values_and_many_rows(dtype):
+    """Negative zero, infinities, NaN, the smallest subnormal and the largest finite value of the
+    16-bit type; and enough rows (66000) that the general row kernel with 16-bit counters runs."""
+    require_gpu()
+    fi = torch.finfo(dtype)
+    tiny_sub = float(torch.tensor(2.0 ** -133 if dtype == torch.bfloat16 else 2.0 ** -24).to(dtype))
+    assert tiny_sub > 0.0
+    specials = np.array([0.0, -0.0, np.inf, -np.inf, np.nan, tiny_sub, -tiny_sub, fi.max, -fi.max, fi.tiny, 1.0, 1.0,
+                         0.5, 2.0, -1.0, 3.0, 1.0], dtype=np.float32)
+    rng = np.random.default_rng(3)
+    A = np.stack([rng.permutation(specials) for _ in range(40)])
+    for alpha, beta in ((0.4, 0.3), (1.0, 1.0), (0.1, 0.1)):
+        view, A16 = _sixteen_bit(A, dtype)
+        S_o, f_o = oracle.select(A16, alpha, beta)
+        K = ci.coreinfer_count(beta, A.shape[1])
+        S = torch.full((K,), -1, dtype=torch.int32, device="cuda")
+        f = torch.full((A.shape[1],), -1, dtype=torch.int32, device="cuda")
+        ws = torch.empty(ci.coreinfer_select_workspace_bytes(*A.shape), dtype=torch.uint8, device="cuda")
+        ci.coreinfer_select_core(view, alpha, beta, S, f, ws, T=A.shape[0], d_ff=A.shape[1], ld_act=view.stride(0))
+        ci.coreinfer_workspace_status(ws)
+        np.testing.assert_array_equal(f.cpu().numpy(), f_o)
+        np.testing.assert_array_equal(S.cpu().numpy(), S_o)
+    T, N = 66000, 40
+    A = (rng.integers(-2, 5, size=(T, N)) * 0.5).astype(np.float32)
+    view, A16 = _sixteen_bit(A, dtype)
+    S_o, f_o = oracle.select(A16, 0.4, 0.2)
+    S = torch.full((ci.coreinfer_count(0.2, N),), -1, dtype=torch.int32, device="cuda")
+    f = torch.full((N,), -1, dtype=torch.int32, device="cuda")
+    ws = torch.empty(ci.coreinfer_select_workspace_bytes(T, N), dtype=torch.uint8, device="cuda")
+    ci.coreinfer_select_core(view, 0.4, 0.2, S, f, ws, T=T, d_ff=N, ld_act=view.stride(0))
+    ci.coreinfer_workspace_status(ws)
+    np.testing.assert_array_equal(f.cpu().numpy(), f_o)
+    np.testing.assert_array_equal(S.cpu().numpy(), S_o)
